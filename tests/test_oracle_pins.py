@@ -1,0 +1,361 @@
+"""Pins for the fp64 oracle: every routine is checked against something that is
+not itself -- closed forms, textbook reductions written independently here in
+numpy / pure Python, hand-expanded small cases and brute-force enumeration.
+Chosen so that a dropped term, a wrong sign or index, or a transposed operand
+in the oracle fails at least one of them."""
+import math
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+
+
+def _rand_batch(rng, m, tmax, equal_policies=False):
+    lens = rng.integers(1, tmax + 1, size=m)
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    n = int(off[-1])
+    r = rng.normal(0, 1, n)
+    V = rng.uniform(0, 1, n)
+    lm = rng.normal(-5, 2, n)
+    lp = lm.copy() if equal_policies else lm + rng.normal(0, 0.7, n)
+    return off, r, V, lp, lm
+
+
+def _segments(off):
+    return [(int(off[j]), int(off[j + 1])) for j in range(len(off) - 1)]
+
+
+# ----------------------------------------------------------------- Retrace ---
+
+def test_lambda_zero_is_one_step_td():
+    # lambda = 0 => c = 0 => Delta_t = delta_t and the target is r + gamma V(s').
+    rng = np.random.default_rng(1)
+    off, r, V, lp, lm = _rand_batch(rng, 40, 12)
+    g = 0.93
+    vt, adv, dl = oracle.retrace(off, r, V, lp, lm, g, 0.0)
+    vnext = np.zeros_like(V)
+    for a, b in _segments(off):
+        vnext[a:b - 1] = V[a + 1:b]
+    np.testing.assert_allclose(dl, r + g * vnext - V, rtol=0, atol=1e-14)
+    np.testing.assert_allclose(adv, dl, rtol=0, atol=0)
+    np.testing.assert_allclose(vt, r + g * vnext, rtol=0, atol=1e-14)
+
+
+def test_on_policy_lambda_one_is_discounted_mc_return():
+    # pi = mu, lambda = 1, V(s_{H+1}) = 0: the target telescopes to
+    # G_t = sum_k gamma^(k-t) r_k (Section 5.1's Monte-Carlo return).
+    rng = np.random.default_rng(2)
+    off, r, V, lp, lm = _rand_batch(rng, 30, 15, equal_policies=True)
+    g = 0.9
+    vt, adv, _ = oracle.retrace(off, r, V, lp, lm, g, 1.0)
+    G = np.zeros_like(r)
+    for a, b in _segments(off):
+        for t in range(a, b):
+            G[t] = sum(g ** (k - t) * r[k] for k in range(t, b))
+    np.testing.assert_allclose(vt, G, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(adv, G - V, rtol=0, atol=1e-12)
+
+
+def test_on_policy_is_gae():
+    # pi = mu: Delta_t = sum_k (gamma lambda)^(k-t) delta_k (textbook GAE).
+    rng = np.random.default_rng(3)
+    off, r, V, lp, lm = _rand_batch(rng, 25, 20, equal_policies=True)
+    g, lam = 0.97, 0.8
+    _, adv, dl = oracle.retrace(off, r, V, lp, lm, g, lam)
+    for a, b in _segments(off):
+        for t in range(a, b):
+            want = sum((g * lam) ** (k - t) * dl[k] for k in range(t, b))
+            assert abs(adv[t] - want) < 1e-12
+
+
+def test_vanishing_ratio_cuts_the_trace():
+    # pi/mu = e^-80 everywhere: c ~ 0 and only the one-step error survives.
+    rng = np.random.default_rng(4)
+    off, r, V, lp, lm = _rand_batch(rng, 20, 10)
+    lp = lm - 80.0
+    _, adv, dl = oracle.retrace(off, r, V, lp, lm, 0.99, 0.95)
+    np.testing.assert_allclose(adv, dl, rtol=0, atol=1e-30)
+
+
+def test_constant_inputs_geometric_series():
+    # V = 0, r = 1, pi = mu: delta = 1 and Delta_t = (1 - (gamma lambda)^n)/(1 - gamma lambda),
+    # n = number of steps from t to the end of its trajectory.
+    lens = [1, 2, 5, 9, 64]
+    off = np.concatenate([[0], np.cumsum(lens)])
+    n = int(off[-1])
+    g, lam = 0.95, 0.9
+    z = np.zeros(n)
+    _, adv, dl = oracle.retrace(off, np.ones(n), z, z, z, g, lam)
+    assert np.all(dl == 1.0)
+    x = g * lam
+    for a, b in _segments(off):
+        for t in range(a, b):
+            assert abs(adv[t] - (1 - x ** (b - t)) / (1 - x)) < 1e-12
+
+
+def test_three_step_hand_expansion_uses_next_steps_trace():
+    # One trajectory of three steps, written out term by term.  The trace that
+    # multiplies delta_k carries c_{t+1}..c_k: the first step's own ratio never
+    # appears, ratios above one are truncated, below one are kept.
+    r = np.array([0.5, -1.0, 2.0])
+    V = np.array([0.3, 0.7, 0.2])
+    lp = np.array([-1.0, -2.0, -1.0])
+    lm = np.array([-3.0, -1.5, -2.0])      # rho = e^2, e^-0.5, e^1
+    g, lam, boot = 0.9, 0.8, 0.4
+    d0 = r[0] + g * V[1] - V[0]
+    d1 = r[1] + g * V[2] - V[1]
+    d2 = r[2] + g * boot - V[2]
+    c1 = lam * min(1.0, math.exp(-0.5))
+    c2 = lam * min(1.0, math.exp(1.0))
+    D2 = d2
+    D1 = d1 + g * c2 * d2
+    D0 = d0 + g * c1 * d1 + g * g * c1 * c2 * d2
+    vt, adv, dl = oracle.retrace([0, 3], r, V, lp, lm, g, lam, bootstrap=[boot])
+    np.testing.assert_allclose(dl, [d0, d1, d2], atol=1e-15)
+    np.testing.assert_allclose(adv, [D0, D1, D2], atol=1e-15)
+    np.testing.assert_allclose(vt, V + np.array([D0, D1, D2]), atol=1e-15)
+    # changing the first step's ratio changes nothing
+    lp2 = lp.copy(); lp2[0] = -7.0
+    _, adv2, _ = oracle.retrace([0, 3], r, V, lp2, lm, g, lam, bootstrap=[boot])
+    np.testing.assert_array_equal(adv, adv2)
+
+
+def test_double_sum_equals_recursion():
+    rng = np.random.default_rng(5)
+    off, r, V, lp, lm = _rand_batch(rng, 12, 64)
+    boot = rng.uniform(0, 1, len(off) - 1)
+    for g, lam in [(0.99, 0.95), (1.0, 1.0), (0.5, 0.3)]:
+        _, adv, _ = oracle.retrace(off, r, V, lp, lm, g, lam, bootstrap=boot)
+        ds = oracle.retrace_double_sum(off, r, V, lp, lm, g, lam, bootstrap=boot)
+        np.testing.assert_allclose(adv, ds, rtol=1e-12, atol=1e-12)
+
+
+def test_trajectories_are_independent():
+    # Permuting trajectories permutes outputs; splitting the batch changes nothing;
+    # zero-length trajectories contribute nothing.
+    rng = np.random.default_rng(6)
+    off, r, V, lp, lm = _rand_batch(rng, 17, 9)
+    g, lam = 0.95, 0.95
+    base = oracle.retrace(off, r, V, lp, lm, g, lam)
+    segs = _segments(off)
+    perm = rng.permutation(len(segs))
+    order = np.concatenate([np.arange(*segs[j]) for j in perm])
+    off_p = np.concatenate([[0], np.cumsum([segs[j][1] - segs[j][0] for j in perm])])
+    out_p = oracle.retrace(off_p, r[order], V[order], lp[order], lm[order], g, lam)
+    for x, y in zip(base, out_p):
+        np.testing.assert_array_equal(x[order], y)
+    cut = 8
+    a = oracle.retrace(off[:cut + 1], r[:off[cut]], V[:off[cut]], lp[:off[cut]], lm[:off[cut]], g, lam)
+    b = oracle.retrace(off[cut:] - off[cut], r[off[cut]:], V[off[cut]:], lp[off[cut]:], lm[off[cut]:], g, lam)
+    for x, ya, yb in zip(base, a, b):
+        np.testing.assert_array_equal(x, np.concatenate([ya, yb]))
+    off_z = np.sort(np.concatenate([off, off[[0, 3, 3, 9, -1]]]))
+    z = oracle.retrace(off_z, r, V, lp, lm, g, lam)
+    for x, y in zip(base, z):
+        np.testing.assert_array_equal(x, y)
+
+
+def test_bootstrap_enters_only_the_last_step():
+    r = np.array([1.0, 1.0]); V = np.array([0.0, 0.0]); z = np.zeros(2)
+    _, _, d0 = oracle.retrace([0, 2], r, V, z, z, 0.5, 0.0)
+    _, _, d1 = oracle.retrace([0, 2], r, V, z, z, 0.5, 0.0, bootstrap=[4.0])
+    np.testing.assert_array_equal(d0, [1.0, 1.0])
+    np.testing.assert_array_equal(d1, [1.0, 3.0])
+
+
+def test_mc_return_closed_form_and_label():
+    g = 0.9
+    off = [0, 4, 5, 11]
+    r = np.ones(11)
+    G, lab = oracle.mc_return(off, r, g)
+    for a, b in _segments(off):
+        for t in range(a, b):
+            assert abs(G[t] - (1 - g ** (b - t)) / (1 - g)) < 1e-13
+    assert lab.tolist() == [1] * 11
+    G, lab = oracle.mc_return([0, 3], np.array([0.0, -0.01, 0.0]), g)
+    np.testing.assert_allclose(G, [-0.009, -0.01, 0.0], atol=1e-15)
+    assert lab.tolist() == [0, 0, 0]
+    G, lab = oracle.mc_return([0, 3], np.array([-0.01, -0.01, 1.0]), 1.0)
+    np.testing.assert_allclose(G, [0.98, 0.99, 1.0], atol=1e-15)
+    assert lab.tolist() == [1, 1, 1]
+
+
+# ----------------------------------------------------------- token log-prob ---
+
+def test_token_logp():
+    tok = np.array([-0.5, -0.25, -1.0, -2.0, -0.125, -4.0])
+    sto = [0, 1, 3, 3, 6]
+    np.testing.assert_array_equal(oracle.token_logp(sto, tok), [-0.5, -1.25, 0.0, -6.125])
+    # single-token steps: the step's log-prob is the token
+    np.testing.assert_array_equal(oracle.token_logp(np.arange(7), tok), tok)
+    # bf16 widening is exact: 0x3F80 = 1.0, 0xBE80 = -0.25, 0x3DCD ~ 0.100098
+    np.testing.assert_array_equal(oracle.bf16_bits_to_f64(np.array([0x3F80, 0xBE80, 0x3DCD], dtype=np.uint16)),
+                                  [1.0, -0.25, 0.10009765625])
+
+
+# ---------------------------------------------------------------- priority ---
+
+def test_priority_hand_values():
+    d = np.array([-2.0, 0.5, 0.0, 3.0])
+    lp = np.array([-1.0, -1.0, -2.0, 0.0])
+    lm = np.array([-1.0, -3.0, -1.0, -0.5])       # rho = 1, e^2 (clipped at 2), e^-1, e^0.5
+    ent = np.array([0.3, 1.0, 2.0, 0.0])
+    w1, w2, w3, clip = 1.0, 0.5, 0.1, 2.0
+    p = np.array([2.0 + 0.5 * 1.0 + 0.03,
+                  0.5 + 0.5 * 2.0 + 0.1,
+                  0.0 + 0.5 * math.exp(-1.0) + 0.2,
+                  3.0 + 0.5 * math.exp(0.5) + 0.0])
+    np.testing.assert_allclose(oracle.priority_mass(d, lp, lm, ent, w1, w2, w3, clip, 1.0), p, rtol=1e-15)
+    np.testing.assert_allclose(oracle.priority_mass(d, lp, lm, ent, w1, w2, w3, clip, 0.5), np.sqrt(p), rtol=1e-15)
+    # only the TD term: |delta|
+    np.testing.assert_array_equal(oracle.priority_mass(d, lp, lm, ent, 1.0, 0.0, 0.0, clip, 1.0), np.abs(d))
+    # clip inactive when large
+    big = oracle.priority_mass(d, lp, lm, ent, 0.0, 1.0, 0.0, 100.0, 1.0)
+    np.testing.assert_allclose(big, np.exp(lp - lm), rtol=1e-15)
+    # no entropy array: the paper's surrogate H_t = -log pi(a_t|s_t)
+    np.testing.assert_allclose(oracle.priority_mass(d, lp, lm, None, 0.0, 0.0, 1.0, clip, 1.0), -lp, rtol=1e-15)
+
+
+def test_trajectory_priority_is_the_mean_of_components():
+    d = np.array([1.0, -3.0, 2.0, 4.0])
+    lp = np.zeros(4); lm = np.array([0.0, math.log(2.0), 0.0, -5.0])   # rho = 1, .5, 1, e^5 -> clip 2
+    ent = np.array([0.2, 0.4, 1.0, 3.0])
+    out = oracle.priority_mass_traj([0, 2, 2, 4], d, lp, lm, ent, 1.0, 0.5, 0.1, 2.0, 1.0)
+    want0 = 2.0 + 0.5 * 0.75 + 0.1 * 0.3
+    want2 = 3.0 + 0.5 * 1.5 + 0.1 * 2.0
+    np.testing.assert_allclose(out, [want0, 0.0, want2], rtol=1e-15)
+    # single-step trajectories: identical to the per-transition priority
+    a = oracle.priority_mass_traj(np.arange(5), d, lp, lm, ent, 1.0, 0.5, 0.1, 2.0, 0.5)
+    b = oracle.priority_mass(d, lp, lm, ent, 1.0, 0.5, 0.1, 2.0, 0.5)
+    np.testing.assert_array_equal(a, b)
+
+
+def test_quantiser_table():
+    S = 2.0 ** 20
+    m = np.array([0.0, -1.0, np.nan, 2.0 ** -21, 1.5 / S, 2.5 / S, 3.5 / S, 1.0, 4095.999, 4096.0,
+                  1e30, np.inf, 2.0 ** -30], dtype=np.float32)
+    q = oracle.quantise(m, S)
+    want = [1, 1, 1, 1, 2, 2, 4, 1 << 20, int(np.rint(np.float64(np.float32(4095.999)) * S)),
+            2 ** 32 - 1, 2 ** 32 - 1, 2 ** 32 - 1, 1]
+    assert q.tolist() == want
+    assert q.dtype == np.uint32
+
+
+def test_prefix_total_and_monotone():
+    rng = np.random.default_rng(7)
+    q = rng.integers(1, 2 ** 32, size=1000, dtype=np.uint64).astype(np.uint32)
+    C, total = oracle.prefix(q)
+    assert total == sum(int(x) for x in q) and total > 2 ** 32
+    assert int(C[-1]) == total
+    assert np.all(np.diff(C.astype(object)) > 0)
+    run = 0
+    for i in range(1000):
+        run += int(q[i])
+        assert int(C[i]) == run
+
+
+# ---------------------------------------------------------------- sampling ---
+
+def _u_for_y(y, total):
+    """Smallest 0.64 fixed-point u whose threshold floor(u total / 2^64) is y."""
+    return -((-y * (1 << 64)) // total)
+
+
+def test_sampling_brute_force_frequencies():
+    # Enumerate every threshold y in [0, total): index i must be hit exactly q_i times.
+    q = np.array([3, 1, 7, 1, 1, 12, 5], dtype=np.uint32)
+    total = int(q.sum())
+    us = np.array([_u_for_y(y, total) for y in range(total)], dtype=np.uint64)
+    for y, u in zip(range(total), us):
+        assert (int(u) * total) >> 64 == y
+    idx = oracle.sample_linear(q, us)
+    counts = np.bincount(idx, minlength=len(q))
+    assert counts.tolist() == q.tolist()
+    assert np.all(np.diff(idx) >= 0)                       # monotone in u
+    # interval form: y -> i  iff  C_{i-1} <= y < C_i
+    C = np.cumsum(q)
+    for y, i in zip(range(total), idx):
+        assert (C[i - 1] if i else 0) <= y < C[i]
+
+
+def test_sampling_extremes_and_large_total():
+    rng = np.random.default_rng(8)
+    q = rng.integers(2 ** 31, 2 ** 32, size=64, dtype=np.uint64).astype(np.uint32)
+    idx = oracle.sample_linear(q, np.array([0, 2 ** 64 - 1, 2 ** 63], dtype=np.uint64))
+    assert idx[0] == 0 and idx[1] == 63
+    C = np.cumsum(q.astype(object))
+    y = (2 ** 63 * int(C[-1])) >> 64
+    assert (C[idx[2] - 1] if idx[2] else 0) <= y < C[idx[2]]
+
+
+def test_is_weights_closed_forms():
+    q = np.full(50, 1234, dtype=np.uint32)
+    idx = np.array([0, 7, 49, 7])
+    np.testing.assert_allclose(oracle.is_weights(q, idx, 0.4, True), 1.0, rtol=1e-15)
+    np.testing.assert_allclose(oracle.is_weights(q, idx, 0.4, False), 1.0, rtol=1e-15)
+    rng = np.random.default_rng(9)
+    q = rng.integers(1, 10 ** 6, size=200).astype(np.uint32)
+    idx = rng.integers(0, 200, size=32)
+    np.testing.assert_allclose(oracle.is_weights(q, idx, 0.0, False), 1.0, rtol=0)
+    beta = 0.6
+    raw = oracle.is_weights(q, idx, beta, False)
+    P = q[idx].astype(np.float64) / float(q.sum(dtype=np.uint64))
+    np.testing.assert_allclose(raw * (200 * P) ** beta, 1.0, rtol=1e-13)
+    nrm = oracle.is_weights(q, idx, beta, True)
+    assert nrm.max() == 1.0
+    assert np.argmax(nrm) == np.argmin(q[idx])            # the rarest sample weighs most
+    np.testing.assert_allclose(nrm, (q[idx] / q[idx].min()) ** -beta, rtol=1e-13)
+    # exact small case: N=2, q=(1,3), beta=1: weights (N P)^-1 = (2, 2/3)
+    np.testing.assert_allclose(oracle.is_weights(np.array([1, 3], dtype=np.uint32), [0, 1], 1.0, False),
+                               [2.0, 2.0 / 3.0], rtol=1e-15)
+
+
+def test_update_sequential_last_wins_and_equals_rebuild():
+    S = 2.0 ** 20
+    n = 16
+    q = np.full(n, 5, dtype=np.uint32)
+    lp = np.zeros(n); lm = np.zeros(n); ent = np.zeros(n)
+    idx = np.array([3, 9, 3, 15])
+    nd = np.array([1.0, 4.0, 9.0, 0.0])
+    mass = oracle.update(q, idx, nd, lp, lm, ent, 1.0, 0.0, 0.0, 2.0, 0.5, S)
+    np.testing.assert_allclose(mass, [1.0, 2.0, 3.0, 0.0])
+    want = np.full(n, 5, dtype=np.uint32)
+    want[3] = 3 << 20; want[9] = 2 << 20; want[15] = 1
+    np.testing.assert_array_equal(q, want)
+    # the integer half alone, fed the same masses, lands in the same state
+    q2 = np.full(n, 5, dtype=np.uint32)
+    oracle.update_from_mass(q2, idx, mass.astype(np.float32), S)
+    np.testing.assert_array_equal(q2, want)
+    # total moved by exactly the winners' differences
+    _, tot = oracle.prefix(q)
+    assert tot == 5 * n + (3 << 20) - 5 + (2 << 20) - 5 + 1 - 5
+
+
+def test_sampling_frequency_tracks_mass_after_update():
+    # After an update the linear scan must see the new masses: enumerate again.
+    q = np.array([2, 2, 2, 2], dtype=np.uint32)
+    oracle.update_from_mass(q, [1], np.array([6.0], dtype=np.float32), 1.0)
+    total = int(q.sum())
+    us = np.array([_u_for_y(y, total) for y in range(total)], dtype=np.uint64)
+    assert np.bincount(oracle.sample_linear(q, us), minlength=4).tolist() == [2, 6, 2, 2]
+
+
+def test_exact_rational_check_of_small_retrace():
+    # pi = mu (c = lambda) with dyadic inputs: compare against exact rational arithmetic.
+    g, lam = Fraction(3, 4), Fraction(1, 2)
+    r = [Fraction(1), Fraction(0), Fraction(-2), Fraction(5, 2)]
+    V = [Fraction(1, 2), Fraction(1, 4), Fraction(3, 4), Fraction(1, 8)]
+    off = [0, 3, 4]
+    want = []
+    for a, b in [(0, 3), (3, 4)]:
+        for t in range(a, b):
+            s = Fraction(0)
+            for k in range(t, b):
+                vn = V[k + 1] if k + 1 < b else Fraction(0)
+                s += (g * lam) ** (k - t) * (r[k] + g * vn - V[k])
+            want.append(s)
+    z = np.zeros(4)
+    _, adv, _ = oracle.retrace(off, [float(x) for x in r], [float(x) for x in V], z, z, float(g), float(lam))
+    assert [Fraction(x) for x in adv] == want
