@@ -1,0 +1,230 @@
+/*
+ * distrl.h -- C ABI of the B200 (sm_100a) learner hot path of DistRL's A-RIDE
+ * algorithm (arXiv 2410.14803): Retrace(lambda) value targets and advantages
+ * (Section 5.2), the DPER replay priority (Section 5.3) and prioritized
+ * proportional sampling with importance-sampling weights and incremental
+ * priority refresh (Section 5.3 and App. A, "Priority-Based Sampling in DPER").
+ *
+ * General rules, valid for every entry point unless it says otherwise:
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  The library
+ *     neither allocates nor frees device memory, and keeps no pointer beyond
+ *     what a sampler handle documents.  Parameter structs (distrl_batch,
+ *     distrl_prio_cfg) and handles live in HOST memory.
+ *   - Arrays are dense and contiguous.  fp32 / uint32 arrays need 4-byte
+ *     alignment, 64-bit arrays 8-byte alignment; 16-byte alignment of every
+ *     array enables the 128-bit load/store path (what torch allocations give).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls enqueue work and return without synchronising.
+ *   - Return value: DISTRL_OK (0) or a negative distrl_status.  Nothing throws,
+ *     aborts or traps.  Problems that only the device can see (bad offsets, an
+ *     index out of range, a bounded wait that ran out) are recorded in the
+ *     status word at the start of the workspace: read it with
+ *     distrl_get_status().
+ *   - Sizes of zero (n = 0, k = 0) are valid and do nothing.
+ *   - There is no CPU fallback: without a CUDA device every compute entry
+ *     point returns DISTRL_ERR_CUDA.
+ */
+#ifndef DISTRL_H
+#define DISTRL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DISTRL_OK = 0,
+    DISTRL_ERR_NULL = -1,      /* a required pointer is NULL                                */
+    DISTRL_ERR_SIZE = -2,      /* negative size, n > DISTRL_MAX_N, struct_size mismatch     */
+    DISTRL_ERR_ALIGN = -3,     /* a pointer breaks its element alignment                    */
+    DISTRL_ERR_WORKSPACE = -4, /* workspace too small or not 256-byte aligned               */
+    DISTRL_ERR_CUDA = -5,      /* a CUDA runtime call failed (see distrl_last_cuda_error)   */
+    DISTRL_ERR_TIMEOUT = -6,   /* device status: a bounded inter-block wait ran out         */
+    DISTRL_ERR_PARAM = -7,     /* gamma/lambda outside [0,1], alpha < 0, scale <= 0, NaN    */
+    DISTRL_ERR_OFFSETS = -8,   /* device status: offsets decreasing, [0] != 0 or [M] != N   */
+    DISTRL_ERR_INDEX = -9      /* device status: a sampled/updated index outside [0, n)     */
+} distrl_status;
+
+#define DISTRL_MAX_N ((int64_t)1 << 33) /* largest transition / token count accepted */
+
+/* ---------------------------------------------------------------------------
+ * The trajectory buffer: N transitions of M trajectories stored flat,
+ * structure-of-arrays.  Trajectory j (Section 3: tau = {(s_t,a_t,r_t,s_t+1)})
+ * owns the flat indices [traj_offsets[j], traj_offsets[j+1]); empty
+ * trajectories are allowed.  Either the per-step action log-probs are given
+ * (logp_*), or, token-level, step t owns the tokens
+ * [step_token_offsets[t], step_token_offsets[t+1]) of two bf16 arrays whose
+ * per-step sums are the action log-probs (the quantity the ratio
+ * rho_t = pi(a_t|s_t)/mu(a_t|s_t) of Section 5.1 needs).
+ * ------------------------------------------------------------------------- */
+typedef struct {
+    uint32_t struct_size;                    /* sizeof(distrl_batch)                       */
+    uint32_t reserved;                       /* 0                                          */
+    int64_t n_transitions;                   /* N                                          */
+    int64_t n_trajectories;                  /* M                                          */
+    const int64_t *traj_offsets;             /* [M+1] non-decreasing, [0] = 0, [M] = N     */
+    const float *rewards;                    /* [N] r_t                                    */
+    const float *values;                     /* [N] V(s_t)                                 */
+    const float *bootstrap_values;           /* [M] V(state after the last step); NULL = 0 */
+    const float *logp_target;                /* [N] log pi(a_t|s_t); NULL if token-level   */
+    const float *logp_behaviour;             /* [N] log mu(a_t|s_t); NULL if token-level   */
+    const int64_t *step_token_offsets;       /* [N+1] or NULL; [0] = 0, non-decreasing     */
+    const uint16_t *tok_logp_target_bf16;    /* [n_tok] bf16 bit patterns                  */
+    const uint16_t *tok_logp_behaviour_bf16; /* [n_tok] bf16 bit patterns                  */
+} distrl_batch;
+
+/* Bytes of workspace distrl_retrace_targets needs for N transitions (any M). */
+size_t distrl_retrace_workspace_bytes(int64_t n_transitions);
+
+/* Zero a workspace's status word.  Call once after allocating a workspace
+ * (retrace or sampler) and before its first use; the status word is sticky
+ * until distrl_get_status() reads it. */
+int distrl_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Retrace(lambda) targets, Section 5.2, with the TD error of App. A:
+ *   rho_t = exp(logpi_t - logmu_t),  c_t = lambda min(1, rho_t)
+ *   delta_t = r_t + gamma V(s_{t+1}) - V(s_t)
+ *   Delta_t = sum_{k>=t} gamma^(k-t) (prod_{i=t+1..k} c_i) delta_k   (per trajectory)
+ *   v_target_t = V(s_t) + Delta_t;  advantage_t = Delta_t;  td_delta_t = delta_t
+ * V(s_{t+1}) of a trajectory's last step is bootstrap_values[j], or 0.
+ * Computed in fp32 as a segmented reverse scan; results agree with fp64
+ * evaluation of the definition to 1e-4 (1 + |ref|).
+ *   v_target, advantage : [N] outputs, required.
+ *   td_delta            : [N] output or NULL.
+ *   logp_target_out, logp_behaviour_out : [N] outputs or NULL; the per-step
+ *       log-probs used (the token sums in token-level mode, a copy otherwise).
+ *   workspace : >= distrl_retrace_workspace_bytes(N) bytes, 256-byte aligned,
+ *       initialised once by distrl_workspace_init; contents are scratch, it
+ *       may be reused by the next call on the same stream, not concurrently.
+ * Outputs must not alias inputs.  Offsets are validated on the device
+ * (DISTRL_ERR_OFFSETS in the status word; outputs are then unspecified but
+ * every access stays in bounds).  Non-finite inputs give unspecified values
+ * inside their own trajectory only.
+ */
+int distrl_retrace_targets(const distrl_batch *batch, float gamma, float lambda,
+                           float *v_target, float *advantage, float *td_delta,
+                           float *logp_target_out, float *logp_behaviour_out,
+                           void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Monte-Carlo return of Section 5.1, G_t = sum_{k>=t} gamma^(k-t) r_k per
+ * trajectory, and the label I[G_t > 0] the state-value classifier is trained
+ * on.  Same scan as above with coefficient gamma and increment r_t.
+ *   mc_return : [N] output or NULL;  label : [N] bytes (0/1) output or NULL.
+ * Only traj_offsets, rewards and the sizes of `batch` are read.
+ */
+int distrl_mc_returns(const distrl_batch *batch, float gamma, float *mc_return,
+                      uint8_t *label, void *workspace, size_t workspace_bytes,
+                      void *stream);
+
+/* ---------------------------------------------------------------------------
+ * DPER priority, Section 5.3, evaluated per transition:
+ *   p_t = w_td |delta_t| + w_rho min(rho_t, rho_clip) + w_ent H_t
+ *   H_t = entropy[t], or -logpi_t when entropy is NULL (the paper's H_t)
+ *   mass_t = p_t^alpha            (App. A: P(i) = p_i^alpha / sum_j p_j^alpha)
+ *   q_t = Q(mass_t): x = (double)mass_t * scale; q = 1 if not (x > 0);
+ *         q = 2^32-1 if x >= 2^32-1; else max(1, round-half-even(x)).
+ * The fixed-point q is what the sampler sums; the floor of 1 keeps every
+ * transition reachable.
+ * ------------------------------------------------------------------------- */
+typedef struct {
+    float w_td, w_rho, w_ent; /* w1, w2, w3 of Section 5.3                    */
+    float rho_clip;           /* upper clip of the ratio term                  */
+    float alpha;              /* prioritisation exponent (0.5 in the paper)    */
+    float scale;              /* fixed-point scale, e.g. 2^20                  */
+} distrl_prio_cfg;
+
+/*  td_delta, logp_target, logp_behaviour : [n] inputs; entropy : [n] or NULL.
+ *  prio_mass : [n] fp32 output or NULL;  prio_q : [n] uint32 output, required.
+ *  prio_q[t] equals Q(prio_mass[t]) exactly. */
+int distrl_compute_priorities(int64_t n, const float *td_delta, const float *logp_target,
+                              const float *logp_behaviour, const float *entropy,
+                              const distrl_prio_cfg *cfg, float *prio_mass,
+                              uint32_t *prio_q, void *stream);
+
+/*
+ * Trajectory-level priority exactly as Section 5.3 writes it: the same formula
+ * applied to the trajectory means of |delta|, min(rho, rho_clip) and H.
+ *   prio_mass : [M] or NULL;  prio_q : [M] required.  Empty trajectory: q = 1.
+ */
+int distrl_compute_priorities_traj(int64_t n, int64_t m, const int64_t *traj_offsets,
+                                   const float *td_delta, const float *logp_target,
+                                   const float *logp_behaviour, const float *entropy,
+                                   const distrl_prio_cfg *cfg, float *prio_mass,
+                                   uint32_t *prio_q, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * Prioritized sampling.  The sampler is a radix tree of exact uint64 partial
+ * sums over prio_q (leaf groups of 128 masses, fan-out 32 above) kept in the
+ * caller's workspace.  Integer sums are associative, so a draw returns exactly
+ * the index a linear scan of cumulative masses returns.
+ * ------------------------------------------------------------------------- */
+typedef struct distrl_sampler distrl_sampler; /* small host-side handle */
+
+size_t distrl_sampler_workspace_bytes(int64_t n);
+
+/*  prio_q : [n] masses; the sampler keeps this pointer, reads it when
+ *      sampling and overwrites entries in distrl_update_priorities.
+ *  workspace : >= distrl_sampler_workspace_bytes(n), 256-byte aligned,
+ *      initialised once by distrl_workspace_init; owned by the caller, must
+ *      outlive the handle.  *out receives a host handle (free it with
+ *      distrl_destroy_sampler; that frees no device memory). */
+int distrl_build_sampler(uint32_t *prio_q, int64_t n, void *workspace,
+                         size_t workspace_bytes, void *stream, distrl_sampler **out);
+
+/*
+ * k independent draws with replacement, P(i) = q_i / total (App. A).
+ *   u_fix : [k] 0.64 fixed-point uniforms (u / 2^64 in [0,1)), device.
+ *   Draw j: y = floor(u_j * total / 2^64); idx_j = min{ i : q_0+..+q_i > y }.
+ *   idx_out : [k] int64, required.
+ *   is_weight_out : [k] fp32 or NULL: w_j = (n q_idx / total)^(-beta)
+ *       (importance-sampling weight of prioritized replay, the definition the
+ *       paper's replay cites); divided by the batch maximum if normalise != 0.
+ */
+int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k, float beta,
+                  int normalise, int64_t *idx_out, float *is_weight_out, void *stream);
+
+/*
+ * Priority refresh for sampled indices (Section 5.3: priorities are updated
+ * from the latest policy).  For j = 0..k-1 in order:
+ *   mass_j = (w_td |new_abs_delta[j]| + w_rho min(rho_i, rho_clip) + w_ent H_i)^alpha,
+ *   i = idx[j], rho_i and H_i gathered from the full [n] arrays;
+ *   q[i] = Q(mass_j); every partial sum of the tree is repaired exactly.
+ * If an index occurs more than once the highest position wins, as a
+ * sequential loop would leave it.
+ *   mass_out : [k] or NULL, the fp32 mass computed for each position.
+ * An index outside [0, n) is skipped and DISTRL_ERR_INDEX recorded.
+ */
+int distrl_update_priorities(distrl_sampler *s, const int64_t *idx, int64_t k,
+                             const float *new_abs_delta, const float *logp_target,
+                             const float *logp_behaviour, const float *entropy,
+                             const distrl_prio_cfg *cfg, float *mass_out, void *stream);
+
+/* Writes total = sum_i q_i to *total_out_device (a device uint64). */
+int distrl_sampler_total(distrl_sampler *s, uint64_t *total_out_device, void *stream);
+
+/* Tree geometry, for inspection: level 1 holds the sums of 128 consecutive
+ * masses, level l+1 the sums of 32 consecutive level-l entries; the top level
+ * has at most 32 entries.  Returns the number of levels; for 1 <= level <=
+ * levels also the byte offset of that level inside the workspace and its
+ * entry count (uint64 entries). */
+int distrl_sampler_level(const distrl_sampler *s, int level, size_t *offset_bytes,
+                         int64_t *count);
+
+int distrl_destroy_sampler(distrl_sampler *s);
+
+/* Synchronises `stream`, returns the workspace's status word (DISTRL_OK or the
+ * first device-side error recorded since the last read) and clears it. */
+int distrl_get_status(void *workspace, void *stream);
+
+const char *distrl_error_string(int code);
+const char *distrl_last_cuda_error(void); /* text of the last failed CUDA call, this thread */
+const char *distrl_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DISTRL_H */

@@ -1,0 +1,257 @@
+"""Thin ctypes binding of the C ABI declared in include/distrl.h.
+
+Argument marshalling only: every function here has the name of the entry point
+it calls, takes torch CUDA tensors (device memory) and passes their pointers on.
+No arithmetic of the method happens in Python, and there is no fallback: if the
+CUDA library cannot be loaded or a call fails, a DistrlError is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+_lib = None
+
+
+class DistrlError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = "%s failed: %d" % (where, code)
+        try:
+            lib = _load()
+            msg = "%s failed: %s (%d)" % (where, lib.distrl_error_string(code).decode(), code)
+            if code == ERR_CUDA:
+                msg += " -- " + lib.distrl_last_cuda_error().decode()
+        except Exception:  # pragma: no cover
+            pass
+        super().__init__(msg)
+
+
+OK, ERR_NULL, ERR_SIZE, ERR_ALIGN, ERR_WORKSPACE, ERR_CUDA = 0, -1, -2, -3, -4, -5
+ERR_TIMEOUT, ERR_PARAM, ERR_OFFSETS, ERR_INDEX = -6, -7, -8, -9
+
+
+class distrl_batch(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+        ("n_transitions", ctypes.c_int64), ("n_trajectories", ctypes.c_int64),
+        ("traj_offsets", ctypes.c_void_p), ("rewards", ctypes.c_void_p), ("values", ctypes.c_void_p),
+        ("bootstrap_values", ctypes.c_void_p), ("logp_target", ctypes.c_void_p),
+        ("logp_behaviour", ctypes.c_void_p), ("step_token_offsets", ctypes.c_void_p),
+        ("tok_logp_target_bf16", ctypes.c_void_p), ("tok_logp_behaviour_bf16", ctypes.c_void_p),
+    ]
+
+
+class distrl_prio_cfg(ctypes.Structure):
+    _fields_ = [("w_td", ctypes.c_float), ("w_rho", ctypes.c_float), ("w_ent", ctypes.c_float),
+                ("rho_clip", ctypes.c_float), ("alpha", ctypes.c_float), ("scale", ctypes.c_float)]
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        path = _build.build()
+    lib = ctypes.CDLL(path)
+    vp, i64, sz, f32, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_float, ctypes.c_int
+    sig = {
+        "distrl_retrace_workspace_bytes": (sz, [i64]),
+        "distrl_workspace_init": (ci, [vp, sz, vp]),
+        "distrl_retrace_targets": (ci, [ctypes.POINTER(distrl_batch), f32, f32, vp, vp, vp, vp, vp, vp, sz, vp]),
+        "distrl_mc_returns": (ci, [ctypes.POINTER(distrl_batch), f32, vp, vp, vp, sz, vp]),
+        "distrl_compute_priorities": (ci, [i64, vp, vp, vp, vp, ctypes.POINTER(distrl_prio_cfg), vp, vp, vp]),
+        "distrl_compute_priorities_traj": (ci, [i64, i64, vp, vp, vp, vp, vp, ctypes.POINTER(distrl_prio_cfg),
+                                                vp, vp, vp]),
+        "distrl_sampler_workspace_bytes": (sz, [i64]),
+        "distrl_build_sampler": (ci, [vp, i64, vp, sz, vp, ctypes.POINTER(vp)]),
+        "distrl_sample": (ci, [vp, vp, i64, f32, ci, vp, vp, vp]),
+        "distrl_update_priorities": (ci, [vp, vp, i64, vp, vp, vp, vp, ctypes.POINTER(distrl_prio_cfg), vp, vp]),
+        "distrl_sampler_total": (ci, [vp, vp, vp]),
+        "distrl_sampler_level": (ci, [vp, ci, ctypes.POINTER(sz), ctypes.POINTER(i64)]),
+        "distrl_destroy_sampler": (ci, [vp]),
+        "distrl_get_status": (ci, [vp, vp]),
+        "distrl_error_string": (ctypes.c_char_p, [ci]),
+        "distrl_last_cuda_error": (ctypes.c_char_p, []),
+        "distrl_version": (ctypes.c_char_p, []),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    _lib = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("expected dtype %s, got %s" % (dtype, t.dtype))
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream or None
+    return int(stream) or None
+
+
+def _check(rc: int, where: str):
+    if rc != OK:
+        raise DistrlError(rc, where)
+
+
+def make_prio_cfg(w_td=1.0, w_rho=0.5, w_ent=0.1, rho_clip=2.0, alpha=0.5, scale=float(2 ** 20)) -> distrl_prio_cfg:
+    return distrl_prio_cfg(w_td, w_rho, w_ent, rho_clip, alpha, scale)
+
+
+def make_batch(traj_offsets, rewards, values, logp_target=None, logp_behaviour=None, bootstrap_values=None,
+               step_token_offsets=None, tok_logp_target=None, tok_logp_behaviour=None) -> distrl_batch:
+    """Fill a distrl_batch from CUDA tensors (kept alive by the caller)."""
+    b = distrl_batch()
+    b.struct_size = ctypes.sizeof(distrl_batch)
+    b.n_transitions = rewards.numel()
+    b.n_trajectories = traj_offsets.numel() - 1
+    b.traj_offsets = _ptr(traj_offsets, torch.int64)
+    b.rewards = _ptr(rewards, torch.float32)
+    b.values = _ptr(values, torch.float32) if values is not None else None
+    b.bootstrap_values = _ptr(bootstrap_values, torch.float32)
+    b.logp_target = _ptr(logp_target, torch.float32)
+    b.logp_behaviour = _ptr(logp_behaviour, torch.float32)
+    b.step_token_offsets = _ptr(step_token_offsets, torch.int64)
+    b.tok_logp_target_bf16 = _ptr(tok_logp_target, torch.bfloat16)
+    b.tok_logp_behaviour_bf16 = _ptr(tok_logp_behaviour, torch.bfloat16)
+    return b
+
+
+def distrl_version() -> str:
+    return _load().distrl_version().decode()
+
+
+def distrl_retrace_workspace_bytes(n: int) -> int:
+    return int(_load().distrl_retrace_workspace_bytes(n))
+
+
+def distrl_sampler_workspace_bytes(n: int) -> int:
+    return int(_load().distrl_sampler_workspace_bytes(n))
+
+
+def distrl_workspace_init(workspace: torch.Tensor, stream=None):
+    _check(_load().distrl_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                         _stream(stream)), "distrl_workspace_init")
+
+
+def distrl_get_status(workspace: torch.Tensor, stream=None) -> int:
+    return int(_load().distrl_get_status(_ptr(workspace), _stream(stream)))
+
+
+def distrl_retrace_targets(batch: distrl_batch, gamma: float, lam: float, v_target, advantage, td_delta=None,
+                           logp_target_out=None, logp_behaviour_out=None, *, workspace, stream=None):
+    _check(_load().distrl_retrace_targets(
+        ctypes.byref(batch), gamma, lam, _ptr(v_target, torch.float32), _ptr(advantage, torch.float32),
+        _ptr(td_delta, torch.float32), _ptr(logp_target_out, torch.float32),
+        _ptr(logp_behaviour_out, torch.float32), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream(stream)), "distrl_retrace_targets")
+
+
+def distrl_mc_returns(batch: distrl_batch, gamma: float, mc_return=None, label=None, *, workspace, stream=None):
+    _check(_load().distrl_mc_returns(
+        ctypes.byref(batch), gamma, _ptr(mc_return, torch.float32), _ptr(label, torch.uint8), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream(stream)), "distrl_mc_returns")
+
+
+def distrl_compute_priorities(td_delta, logp_target, logp_behaviour, entropy, cfg: distrl_prio_cfg, prio_mass,
+                              prio_q, stream=None):
+    _check(_load().distrl_compute_priorities(
+        td_delta.numel(), _ptr(td_delta, torch.float32), _ptr(logp_target, torch.float32),
+        _ptr(logp_behaviour, torch.float32), _ptr(entropy, torch.float32), ctypes.byref(cfg),
+        _ptr(prio_mass, torch.float32), _ptr(prio_q), _stream(stream)), "distrl_compute_priorities")
+
+
+def distrl_compute_priorities_traj(traj_offsets, td_delta, logp_target, logp_behaviour, entropy,
+                                   cfg: distrl_prio_cfg, prio_mass, prio_q, stream=None):
+    _check(_load().distrl_compute_priorities_traj(
+        td_delta.numel(), traj_offsets.numel() - 1, _ptr(traj_offsets, torch.int64),
+        _ptr(td_delta, torch.float32), _ptr(logp_target, torch.float32), _ptr(logp_behaviour, torch.float32),
+        _ptr(entropy, torch.float32), ctypes.byref(cfg), _ptr(prio_mass, torch.float32), _ptr(prio_q),
+        _stream(stream)), "distrl_compute_priorities_traj")
+
+
+class Sampler:
+    """Owns the host handle returned by distrl_build_sampler (frees it on close)."""
+
+    def __init__(self, handle: int, prio_q: torch.Tensor, workspace: torch.Tensor):
+        self.handle = handle
+        self.prio_q = prio_q          # kept alive: the library reads and updates it
+        self.workspace = workspace    # kept alive: holds the tree
+
+    def close(self):
+        if self.handle:
+            _load().distrl_destroy_sampler(self.handle)
+            self.handle = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def distrl_build_sampler(prio_q: torch.Tensor, workspace: torch.Tensor, stream=None) -> Sampler:
+    if prio_q.element_size() != 4:
+        raise ValueError("prio_q must hold 32-bit masses")
+    out = ctypes.c_void_p()
+    _check(_load().distrl_build_sampler(_ptr(prio_q), prio_q.numel(), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream(stream),
+                                        ctypes.byref(out)), "distrl_build_sampler")
+    return Sampler(out.value, prio_q, workspace)
+
+
+def distrl_sample(s: Sampler, u_fix, beta: float, normalise: bool, idx_out, is_weight_out=None, stream=None):
+    if u_fix.element_size() != 8:
+        raise ValueError("u_fix must hold 64-bit fixed-point uniforms")
+    _check(_load().distrl_sample(s.handle, _ptr(u_fix), u_fix.numel(), beta, 1 if normalise else 0,
+                                 _ptr(idx_out, torch.int64), _ptr(is_weight_out, torch.float32),
+                                 _stream(stream)), "distrl_sample")
+
+
+def distrl_update_priorities(s: Sampler, idx, new_abs_delta, logp_target, logp_behaviour, entropy,
+                             cfg: distrl_prio_cfg, mass_out=None, stream=None):
+    _check(_load().distrl_update_priorities(
+        s.handle, _ptr(idx, torch.int64), idx.numel(), _ptr(new_abs_delta, torch.float32),
+        _ptr(logp_target, torch.float32), _ptr(logp_behaviour, torch.float32), _ptr(entropy, torch.float32),
+        ctypes.byref(cfg), _ptr(mass_out, torch.float32), _stream(stream)), "distrl_update_priorities")
+
+
+def distrl_sampler_total(s: Sampler, total_out: torch.Tensor, stream=None):
+    _check(_load().distrl_sampler_total(s.handle, _ptr(total_out), _stream(stream)), "distrl_sampler_total")
+
+
+def distrl_sampler_level(s: Sampler, level: int):
+    """(levels, byte offset of `level` in the workspace, entry count)."""
+    off, cnt = ctypes.c_size_t(0), ctypes.c_int64(0)
+    levels = _load().distrl_sampler_level(s.handle, level, ctypes.byref(off), ctypes.byref(cnt))
+    return int(levels), int(off.value), int(cnt.value)
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A zero-filled, 256-byte aligned device buffer (torch allocations are 512-byte aligned)."""
+    ws = torch.zeros(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    assert ws.data_ptr() % 256 == 0
+    return ws

@@ -1,0 +1,64 @@
+// Shared host/device helpers of the CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "distrl.h"
+
+namespace distrl {
+
+// ---- host-side helpers ------------------------------------------------------
+
+// Records the text of a failed CUDA call for distrl_last_cuda_error().
+int record_cuda_error(cudaError_t e, const char *what);
+
+#define DISTRL_CUDA_TRY(expr)                                              \
+    do {                                                                   \
+        cudaError_t e__ = (expr);                                          \
+        if (e__ != cudaSuccess) return ::distrl::record_cuda_error(e__, #expr); \
+    } while (0)
+
+static inline bool aligned_to(const void *p, size_t a) {
+    return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0;
+}
+static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// Every workspace starts with this header (256 bytes reserved).
+struct WorkspaceHeader {
+    int status;          // sticky device-side status word (distrl_status)
+    unsigned int ticket; // dynamic tile counter of the scan
+    unsigned int qmin;   // batch minimum of sampled masses (sampler)
+    unsigned int done;   // finished-block counter (sampler)
+    unsigned int bad_epoch; // call number whose offsets failed validation (scan)
+};
+constexpr size_t kHeaderBytes = 256;
+
+// ---- device-side helpers ----------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u32(unsigned int *p, unsigned int v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Records the first device-side error; later ones are dropped.
+__device__ __forceinline__ void set_status(int *status, int code) { atomicCAS(status, 0, code); }
+
+// Streaming 128-bit loads/stores: data that is touched once should not evict
+// what the rest of the pass keeps in L2.
+__device__ __forceinline__ float4 ldg_stream_f4(const float *p) {
+    return __ldcs(reinterpret_cast<const float4 *>(p));
+}
+__device__ __forceinline__ void stg_stream_f4(float *p, float4 v) {
+    __stcs(reinterpret_cast<float4 *>(p), v);
+}
+
+#endif // __CUDACC__
+
+} // namespace distrl

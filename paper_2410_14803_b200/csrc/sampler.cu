@@ -1,0 +1,438 @@
+// Prioritized proportional sampling over fixed-point masses (App. A,
+// "Priority-Based Sampling in DPER": P(i) = p_i^alpha / sum_j p_j^alpha) -- sm_100a.
+//
+// Data structure: a radix tree of exact uint64 partial sums over the uint32
+// masses q.  Level 1 entry g = sum of q[128 g .. 128 g + 127]; level l+1 entry
+// g = sum of 32 consecutive level-l entries; the top level has <= 32 entries.
+// Integer addition is associative, so descending the tree returns exactly
+// min{ i : q_0 + .. + q_i > y }, the answer of a linear scan.
+//   build  : one streaming pass over q writes levels 1 and 2, one small block
+//            finishes the levels above;
+//   sample : one warp per draw; per level one coalesced 256-byte load, a
+//            shuffle prefix sum and a ballot;
+//   update : one block; a shared-memory hash table elects, for every distinct
+//            index, the highest batch position (what a sequential loop would
+//            leave), the winners store the new mass and add new - old to every
+//            ancestor, so the tree stays bit-identical to a rebuild.
+#include "priority.cuh"
+
+#include <new>
+
+namespace distrl {
+
+constexpr int kLeaf = 128;      // masses per level-1 entry
+constexpr int kFan = 32;        // fan-out above level 1
+constexpr int kMaxLevels = 8;   // enough for n <= 2^33
+constexpr int kSampleThreads = 256;
+constexpr int kUpdateThreads = 1024;
+constexpr int kUpdateChunk = 8192;              // batch positions per update launch
+constexpr int kHashSlots = 2 * kUpdateChunk;    // load factor <= 0.5
+constexpr int kPosBits = 13;                    // log2(kUpdateChunk)
+constexpr int kAccCap = 2048;                   // tree entries accumulated in shared memory
+
+struct Tree {
+    int levels;                     // sum levels 1..levels
+    int64_t n;
+    int64_t count[kMaxLevels + 1];  // entries of level l (index 0 unused)
+    unsigned long long *lvl[kMaxLevels + 1];
+    uint32_t *q;
+    WorkspaceHeader *hdr;
+};
+
+static size_t tree_layout(int64_t n, void *base, Tree *t, size_t *offsets) {
+    int64_t count[kMaxLevels + 1] = {0};
+    int levels = 1;
+    count[1] = n > 0 ? ceil_div(n, kLeaf) : 1;
+    while (count[levels] > kFan && levels < kMaxLevels) {
+        count[levels + 1] = ceil_div(count[levels], kFan);
+        ++levels;
+    }
+    size_t o = kHeaderBytes;
+    for (int l = 1; l <= levels; ++l) {
+        if (offsets) offsets[l] = o;
+        if (t) t->lvl[l] = reinterpret_cast<unsigned long long *>(static_cast<char *>(base) + o);
+        o = round_up(o + sizeof(unsigned long long) * count[l], 256);
+    }
+    if (t) {
+        t->levels = levels;
+        t->n = n;
+        for (int l = 0; l <= kMaxLevels; ++l) t->count[l] = count[l];
+        t->hdr = reinterpret_cast<WorkspaceHeader *>(base);
+    }
+    return o;
+}
+
+__device__ __forceinline__ unsigned long long warp_incl_scan_u64(unsigned long long v, int lane) {
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        unsigned long long o = __shfl_up_sync(0xffffffffu, v, d);
+        if (lane >= d) v += o;
+    }
+    return v;
+}
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+    return v;
+}
+
+// ---------------------------------------------------------------------------
+// build, pass 1: block b owns level-2 entry b = leaf groups [32 b, 32 b + 32);
+// each of its 8 warps sums 4 leaf groups with the 16 loads issued up front.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) build_leaf_kernel(Tree t, int vec_ok) {
+    __shared__ unsigned long long s_l1[kFan];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        t.hdr->qmin = 0xffffffffu;
+        t.hdr->done = 0u;
+    }
+    const int64_t g0 = (int64_t)blockIdx.x * kFan + warp * 4;
+    unsigned long long s[4];
+    if (vec_ok && (g0 + 4) * kLeaf <= t.n) {
+        uint4 v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            v[i] = __ldg(reinterpret_cast<const uint4 *>(t.q + (g0 + i) * kLeaf + 4 * lane));
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            s[i] = (unsigned long long)v[i].x + v[i].y + v[i].z + v[i].w;
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            int64_t p = (g0 + i) * kLeaf + 4 * lane;
+            s[i] = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (p + e < t.n) s[i] += t.q[p + e];
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        s[i] = warp_sum_u64(s[i]);
+        if (lane == 0) {
+            if (g0 + i < t.count[1]) t.lvl[1][g0 + i] = s[i];
+            s_l1[warp * 4 + i] = (g0 + i < t.count[1]) ? s[i] : 0ull;
+        }
+    }
+    if (t.levels < 2) return;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned long long tot = warp_sum_u64(s_l1[lane]);
+        if (lane == 0 && blockIdx.x < t.count[2]) t.lvl[2][blockIdx.x] = tot;
+    }
+}
+
+// build, pass 2: levels 3.. from level 2, one block.
+__global__ void __launch_bounds__(1024) build_upper_kernel(Tree t) {
+    for (int l = 3; l <= t.levels; ++l) {
+        for (int64_t i = threadIdx.x; i < t.count[l]; i += blockDim.x) {
+            unsigned long long s = 0;
+            for (int e = 0; e < kFan; ++e) {
+                int64_t c = i * kFan + e;
+                if (c < t.count[l - 1]) s += t.lvl[l - 1][c];
+            }
+            t.lvl[l][i] = s;
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void total_kernel(Tree t, unsigned long long *out) {
+    const int lane = threadIdx.x;
+    unsigned long long v = (lane < t.count[t.levels]) ? t.lvl[t.levels][lane] : 0ull;
+    v = warp_sum_u64(v);
+    if (lane == 0) *out = v;
+}
+
+// ---------------------------------------------------------------------------
+// sample: one warp per draw.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ int pick_lane(unsigned long long incl, unsigned long long v, unsigned long long y) {
+    unsigned int mask = __ballot_sync(0xffffffffu, incl > y);
+    if (mask) return __ffs(mask) - 1;
+    // unreachable while y < sum of the children; stay inside the populated part
+    unsigned int nz = __ballot_sync(0xffffffffu, v != 0ull);
+    return nz ? (31 - __clz(nz)) : 0;
+}
+
+__global__ void __launch_bounds__(kSampleThreads) sample_kernel(
+    Tree t, const unsigned long long *__restrict__ u, int64_t k, float beta, int normalise,
+    int64_t *__restrict__ idx_out, float *__restrict__ w_out, int vec_ok) {
+    __shared__ int s_last;
+    const int lane = threadIdx.x & 31;
+    const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (j < k) {
+        // top level: its entries sum to the total mass
+        int l = t.levels;
+        unsigned long long v = (lane < t.count[l]) ? __ldcg(&t.lvl[l][lane]) : 0ull;
+        unsigned long long incl = warp_incl_scan_u64(v, lane);
+        const unsigned long long total = __shfl_sync(0xffffffffu, incl, 31);
+        unsigned long long y = __umul64hi(u[j], total);
+        int64_t node = 0;
+        while (true) {
+            int c = pick_lane(incl, v, y);
+            y -= __shfl_sync(0xffffffffu, incl - v, c);
+            node = node * kFan + c;
+            if (--l == 0) break;
+            int64_t i = node * kFan + lane;
+            v = (i < t.count[l]) ? __ldcg(&t.lvl[l][i]) : 0ull;
+            incl = warp_incl_scan_u64(v, lane);
+        }
+        // leaf group `node`: 128 masses, 4 per lane
+        const int64_t p = node * kLeaf + 4 * lane;
+        uint32_t qv[4];
+        if (vec_ok && p + 3 < t.n) {
+            uint4 x = __ldcg(reinterpret_cast<const uint4 *>(t.q + p));
+            qv[0] = x.x; qv[1] = x.y; qv[2] = x.z; qv[3] = x.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) qv[e] = (p + e < t.n) ? __ldcg(t.q + p + e) : 0u;
+        }
+        v = (unsigned long long)qv[0] + qv[1] + qv[2] + qv[3];
+        incl = warp_incl_scan_u64(v, lane);
+        int c = pick_lane(incl, v, y);
+        y -= __shfl_sync(0xffffffffu, incl - v, c);
+        if (lane == c) {
+            int e = 0;
+            while (e < 3 && y >= qv[e]) { y -= qv[e]; ++e; }
+            int64_t idx = p + e;
+            if (idx >= t.n) { idx = t.n - 1; set_status(&t.hdr->status, DISTRL_ERR_INDEX); }
+            idx_out[j] = idx;
+            if (w_out) {
+                uint32_t qs = qv[e];
+                if (normalise) atomicMin(&t.hdr->qmin, qs);
+                else w_out[j] = powf((float)((double)t.n * (double)qs / (double)total), -beta);
+            }
+        }
+    }
+    if (!(w_out && normalise)) return;
+    // The block that finishes last divides by the batch maximum.  The largest
+    // weight belongs to the smallest sampled mass, so w_j = (q_j / q_min)^-beta.
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        unsigned int done = atomicAdd(&t.hdr->done, 1u);
+        s_last = (done == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const unsigned int qmin = atomicMin(&t.hdr->qmin, 0xffffffffu); // atomic read
+    for (int64_t i = threadIdx.x; i < k; i += blockDim.x) {
+        uint32_t qs = __ldcg(t.q + __ldcg(idx_out + i));
+        w_out[i] = powf((float)((double)qs / (double)qmin), -beta);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) { // ready for the next call
+        t.hdr->qmin = 0xffffffffu;
+        t.hdr->done = 0u;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// update: one block per chunk of <= kUpdateChunk batch positions.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ unsigned int hash_idx(unsigned long long key) {
+    key ^= key >> 33;
+    key *= 0xff51afd7ed558ccdull;
+    key ^= key >> 29;
+    return (unsigned int)key & (kHashSlots - 1);
+}
+
+__global__ void __launch_bounds__(kUpdateThreads) update_kernel(
+    Tree t, const int64_t *__restrict__ idx, int k, const float *__restrict__ new_abs_delta,
+    const float *__restrict__ lp, const float *__restrict__ lm, const float *__restrict__ ent, PrioCfg c,
+    float *__restrict__ mass_out) {
+    extern __shared__ unsigned long long s_mem[];
+    unsigned long long *s_tab = s_mem;             // [kHashSlots] (index + 1) << kPosBits | position
+    unsigned long long *s_acc = s_mem + kHashSlots; // [kAccCap] pending sums for the small top levels
+
+    // which levels accumulate in shared memory (from the top down, while they fit)
+    int acc_from = t.levels + 1; // levels >= acc_from live in s_acc
+    int acc_off[kMaxLevels + 2];
+    {
+        int used = 0;
+        for (int l = t.levels; l >= 1; --l) {
+            if (used + t.count[l] > kAccCap) break;
+            acc_off[l] = used;
+            used += (int)t.count[l];
+            acc_from = l;
+        }
+        for (int i = threadIdx.x; i < used; i += blockDim.x) s_acc[i] = 0ull;
+    }
+    for (int i = threadIdx.x; i < kHashSlots; i += blockDim.x) s_tab[i] = 0ull;
+    __syncthreads();
+
+    // phase 1: per distinct index keep the highest batch position
+    for (int j = threadIdx.x; j < k; j += blockDim.x) {
+        int64_t i = idx[j];
+        if (i < 0 || i >= t.n) { set_status(&t.hdr->status, DISTRL_ERR_INDEX); continue; }
+        const unsigned long long tag = (unsigned long long)(i + 1);
+        const unsigned long long packed = (tag << kPosBits) | (unsigned long long)j;
+        unsigned int h = hash_idx(tag);
+        while (true) {
+            unsigned long long cur = s_tab[h];
+            if (cur == 0ull) {
+                cur = atomicCAS(&s_tab[h], 0ull, packed);
+                if (cur == 0ull) break;
+            }
+            if ((cur >> kPosBits) == tag) { atomicMax(&s_tab[h], packed); break; }
+            h = (h + 1) & (kHashSlots - 1);
+        }
+    }
+    __syncthreads();
+
+    // phase 2: every position computes its mass; the winner applies it
+    for (int j = threadIdx.x; j < k; j += blockDim.x) {
+        int64_t i = idx[j];
+        if (i < 0 || i >= t.n) { if (mass_out) mass_out[j] = 0.f; continue; }
+        float p = lp[i];
+        float mass = prio_mass(new_abs_delta[j], p, lm[i], ent ? ent[i] : -p, c);
+        if (mass_out) mass_out[j] = mass;
+        const unsigned long long tag = (unsigned long long)(i + 1);
+        unsigned int h = hash_idx(tag);
+        unsigned long long cur;
+        while (((cur = s_tab[h]) >> kPosBits) != tag) h = (h + 1) & (kHashSlots - 1);
+        if ((int)(cur & ((1u << kPosBits) - 1u)) != j) continue;
+        const uint32_t qn = prio_quantise(mass, c.scale), qo = t.q[i];
+        if (qn == qo) continue;
+        t.q[i] = qn;
+        const unsigned long long diff = (unsigned long long)qn - (unsigned long long)qo; // mod 2^64
+        int64_t node = i / kLeaf;
+        for (int l = 1; l <= t.levels; ++l) {
+            if (l >= acc_from) atomicAdd(&s_acc[acc_off[l] + (int)node], diff);
+            else atomicAdd(&t.lvl[l][node], diff);
+            node /= kFan;
+        }
+    }
+    __syncthreads();
+    // flush the shared-memory sums: this block is the only writer
+    for (int l = acc_from; l <= t.levels; ++l)
+        for (int i = threadIdx.x; i < t.count[l]; i += blockDim.x) {
+            unsigned long long d = s_acc[acc_off[l] + i];
+            if (d) t.lvl[l][i] += d;
+        }
+}
+
+} // namespace distrl
+
+using namespace distrl;
+
+struct distrl_sampler {
+    Tree tree;
+    size_t offsets[kMaxLevels + 1];
+    int vec_ok;
+};
+
+extern "C" size_t distrl_sampler_workspace_bytes(int64_t n) {
+    if (n < 0) n = 0;
+    return tree_layout(n, nullptr, nullptr, nullptr);
+}
+
+extern "C" int distrl_build_sampler(uint32_t *prio_q, int64_t n, void *workspace, size_t workspace_bytes,
+                                    void *stream, distrl_sampler **out) {
+    if (!out) return DISTRL_ERR_NULL;
+    *out = nullptr;
+    if (n < 0 || n > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
+    if (!workspace || (n > 0 && !prio_q)) return DISTRL_ERR_NULL;
+    if (!aligned_to(prio_q, 4)) return DISTRL_ERR_ALIGN;
+    if (!aligned_to(workspace, 256) || workspace_bytes < tree_layout(n, nullptr, nullptr, nullptr))
+        return DISTRL_ERR_WORKSPACE;
+    distrl_sampler *s = new (std::nothrow) distrl_sampler();
+    if (!s) return DISTRL_ERR_CUDA;
+    tree_layout(n, workspace, &s->tree, s->offsets);
+    s->tree.q = prio_q;
+    s->vec_ok = aligned_to(prio_q, 16) ? 1 : 0;
+    *out = s;
+    if (n == 0) return DISTRL_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const Tree &t = s->tree;
+    unsigned grid = (unsigned)(t.levels >= 2 ? t.count[2] : 1);
+    build_leaf_kernel<<<grid, 256, 0, st>>>(t, s->vec_ok);
+    DISTRL_CUDA_TRY(cudaGetLastError());
+    if (t.levels >= 3) {
+        build_upper_kernel<<<1, 1024, 0, st>>>(t);
+        DISTRL_CUDA_TRY(cudaGetLastError());
+    }
+    return DISTRL_OK;
+}
+
+extern "C" int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k, float beta, int normalise,
+                             int64_t *idx_out, float *is_weight_out, void *stream) {
+    if (!s) return DISTRL_ERR_NULL;
+    if (k < 0 || k > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
+    if (!(beta == beta)) return DISTRL_ERR_PARAM;
+    if (k == 0) return DISTRL_OK;
+    if (s->tree.n == 0) return DISTRL_ERR_SIZE; // nothing to draw from
+    if (!u_fix || !idx_out) return DISTRL_ERR_NULL;
+    if (!aligned_to(u_fix, 8) || !aligned_to(idx_out, 8) || !aligned_to(is_weight_out, 4)) return DISTRL_ERR_ALIGN;
+    const int64_t blocks = ceil_div(k * 32, kSampleThreads);
+    sample_kernel<<<(unsigned)blocks, kSampleThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        s->tree, reinterpret_cast<const unsigned long long *>(u_fix), k, beta, normalise, idx_out, is_weight_out,
+        s->vec_ok);
+    DISTRL_CUDA_TRY(cudaGetLastError());
+    return DISTRL_OK;
+}
+
+extern "C" int distrl_update_priorities(distrl_sampler *s, const int64_t *idx, int64_t k,
+                                        const float *new_abs_delta, const float *lp, const float *lm,
+                                        const float *entropy, const distrl_prio_cfg *cfg, float *mass_out,
+                                        void *stream) {
+    if (!s) return DISTRL_ERR_NULL;
+    if (k < 0 || k > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
+    PrioCfg c;
+    int rc = check_prio_cfg(cfg, &c);
+    if (rc) return rc;
+    if (k == 0) return DISTRL_OK;
+    if (!idx || !new_abs_delta || !lp || !lm) return DISTRL_ERR_NULL;
+    if (!aligned_to(idx, 8) || !aligned_to(new_abs_delta, 4) || !aligned_to(lp, 4) || !aligned_to(lm, 4) ||
+        !aligned_to(entropy, 4) || !aligned_to(mass_out, 4))
+        return DISTRL_ERR_ALIGN;
+    const size_t smem = sizeof(unsigned long long) * (kHashSlots + kAccCap);
+    {   // opt in to the large dynamic shared-memory window, once per device
+        static bool attr_set[64] = {false};
+        int dev = 0;
+        DISTRL_CUDA_TRY(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+            DISTRL_CUDA_TRY(cudaFuncSetAttribute(update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        }
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // chunks run one after another on the stream, so "later position wins" also holds across chunks
+    for (int64_t o = 0; o < k; o += kUpdateChunk) {
+        int kc = (int)((k - o < kUpdateChunk) ? (k - o) : kUpdateChunk);
+        update_kernel<<<1, kUpdateThreads, smem, st>>>(s->tree, idx + o, kc, new_abs_delta + o, lp, lm, entropy, c,
+                                                       mass_out ? mass_out + o : nullptr);
+        DISTRL_CUDA_TRY(cudaGetLastError());
+    }
+    return DISTRL_OK;
+}
+
+extern "C" int distrl_sampler_total(distrl_sampler *s, uint64_t *total_out_device, void *stream) {
+    if (!s || !total_out_device) return DISTRL_ERR_NULL;
+    if (!aligned_to(total_out_device, 8)) return DISTRL_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (s->tree.n == 0) {
+        DISTRL_CUDA_TRY(cudaMemsetAsync(total_out_device, 0, sizeof(uint64_t), st));
+        return DISTRL_OK;
+    }
+    total_kernel<<<1, 32, 0, st>>>(s->tree, reinterpret_cast<unsigned long long *>(total_out_device));
+    DISTRL_CUDA_TRY(cudaGetLastError());
+    return DISTRL_OK;
+}
+
+extern "C" int distrl_sampler_level(const distrl_sampler *s, int level, size_t *offset_bytes, int64_t *count) {
+    if (!s) return DISTRL_ERR_NULL;
+    if (level >= 1 && level <= s->tree.levels) {
+        if (offset_bytes) *offset_bytes = s->offsets[level];
+        if (count) *count = s->tree.count[level];
+    }
+    return s->tree.levels;
+}
+
+extern "C" int distrl_destroy_sampler(distrl_sampler *s) {
+    delete s;
+    return DISTRL_OK;
+}

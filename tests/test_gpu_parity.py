@@ -1,0 +1,358 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle
+on the same seeded inputs.  Bit-exact for masses, partial sums and indices;
+max |err| <= 1e-4 (1 + |ref|) for every fp32 output."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2410_14803_b200 as distrl
+from paper_2410_14803_b200 import synth
+
+from helpers import (TOL, assert_close, check_retrace, dev, gpu_retrace, prio_cfg_of, random_batch, read_tree,
+                     sample_by_prefix, tree_from_q)
+
+pytestmark = pytest.mark.gpu
+
+
+# ------------------------------------------------------------------ Retrace ---
+
+@pytest.mark.parametrize("index", [0, 1, 2, 3])
+def test_retrace_workloads(index):
+    w = synth.make_workload(index)
+    a = w.arrays
+    check_retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"],
+                  w.gamma, w.lam)
+
+
+@pytest.mark.parametrize("kind", ["single", "ones", "tile_aligned", "tile_straddle", "with_empty", "long_mixed"])
+@pytest.mark.parametrize("n", [1, 5, 2048, 2049, 20000, 70001])
+def test_retrace_adversarial_layouts(kind, n):
+    off = synth.adversarial_offsets(kind, n)
+    r, V, lp, lm = random_batch(11 + n, off)
+    check_retrace(off, r, V, lp, lm, 0.99, 0.95)
+
+
+def test_retrace_long_trajectory_many_tiles_on_policy():
+    # One trajectory over ~150 tiles with pi = mu and lambda = gamma = 1: the carry crosses
+    # every tile boundary undamped, so every look-back link matters.
+    n = 300001
+    off = np.array([0, n], dtype=np.int64)
+    rng = np.random.default_rng(5)
+    r = rng.normal(0, 0.01, n).astype(np.float32)
+    V = rng.random(n, dtype=np.float32)
+    lm = rng.normal(-5, 2, n).astype(np.float32)
+    out = gpu_retrace(off, r, V, lm, lm, 1.0, 1.0)
+    assert out["status"] == 0
+    vt, adv, dl = oracle.retrace(off, r, V, lm, lm, 1.0, 1.0)
+    # fp32 running sums over 3e5 terms: compare with a tolerance scaled to the sum of magnitudes
+    bound = 1e-4 * (1.0 + np.abs(adv)) + 2e-7 * np.cumsum(np.abs(dl[::-1]))[::-1] * 8
+    assert np.all(np.abs(out["advantage"] - adv) <= bound)
+
+
+@pytest.mark.parametrize("gamma,lam", [(0.95, 0.0), (1.0, 1.0), (0.0, 0.5), (0.5, 1.0)])
+def test_retrace_parameter_corners(gamma, lam):
+    w = synth.make_workload(1)
+    a = w.arrays
+    check_retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"], gamma, lam)
+
+
+def test_retrace_bootstrap_values():
+    off = synth.adversarial_offsets("with_empty", 9000)
+    r, V, lp, lm = random_batch(3, off)
+    boot = np.random.default_rng(4).random(off.shape[0] - 1, dtype=np.float32)
+    check_retrace(off, r, V, lp, lm, 0.97, 0.9, boot=boot)
+
+
+@pytest.mark.parametrize("n", [3, 4099, 30011])
+def test_retrace_unaligned_pointers_and_ragged_tail(n):
+    off = synth.adversarial_offsets("long_mixed", n)
+    r, V, lp, lm = random_batch(n, off)
+    check_retrace(off, r, V, lp, lm, 0.99, 0.95, misalign=True)
+
+
+def test_retrace_without_optional_outputs_and_copy_of_logp():
+    w = synth.make_workload(1)
+    a = w.arrays
+    out = gpu_retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"],
+                      w.gamma, w.lam, want_delta=False, want_logp=True)
+    vt, adv, _ = oracle.retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"],
+                                a["logp_behaviour"], w.gamma, w.lam)
+    assert_close(out["v_target"], vt, "v_target")
+    np.testing.assert_array_equal(out["logp_target"], a["logp_target"])
+    np.testing.assert_array_equal(out["logp_behaviour"], a["logp_behaviour"])
+
+
+def test_retrace_is_deterministic():
+    w = synth.make_workload(2)
+    a = w.arrays
+    args = (a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"], w.gamma, w.lam)
+    x, y = gpu_retrace(*args), gpu_retrace(*args)
+    for key in ("v_target", "advantage", "td_delta"):
+        np.testing.assert_array_equal(x[key].view(np.uint32), y[key].view(np.uint32))
+
+
+def test_retrace_bad_offsets_are_reported_not_fatal():
+    off = np.array([0, 10, 7, 20], dtype=np.int64)     # decreasing
+    r, V, lp, lm = random_batch(1, np.array([0, 20]))
+    out = gpu_retrace(off, r, V, lp, lm, 0.9, 0.9)
+    assert out["status"] == distrl.binding.ERR_OFFSETS
+    off = np.array([0, 10, 19], dtype=np.int64)        # does not end at N
+    out = gpu_retrace(off, r, V, lp, lm, 0.9, 0.9)
+    assert out["status"] == distrl.binding.ERR_OFFSETS
+    # the workspace stays usable: a valid call afterwards is correct
+    check_retrace(np.array([0, 10, 20], dtype=np.int64), r, V, lp, lm, 0.9, 0.9)
+
+
+def test_mc_returns():
+    for index in (1, 2):
+        w = synth.make_workload(index)
+        a = w.arrays
+        n = w.n
+        t_off, t_r = dev(a["traj_offsets"]), dev(a["rewards"])
+        batch = distrl.make_batch(t_off, t_r, None)
+        G = torch.empty(n, dtype=torch.float32, device="cuda")
+        lab = torch.empty(n, dtype=torch.uint8, device="cuda")
+        ws = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+        distrl.distrl_workspace_init(ws)
+        distrl.distrl_mc_returns(batch, w.gamma, G, lab, workspace=ws)
+        assert distrl.distrl_get_status(ws) == 0
+        Gr, labr = oracle.mc_return(a["traj_offsets"], a["rewards"], w.gamma)
+        assert_close(G.cpu().numpy(), Gr, "mc_return")
+        # the label is decided in fp32 on the device: it must match the sign of the device's own G,
+        # and the oracle's label wherever G is not within rounding of zero
+        np.testing.assert_array_equal(lab.cpu().numpy(), (G.cpu().numpy() > 0).astype(np.uint8))
+        clear = np.abs(Gr) > 1e-5
+        np.testing.assert_array_equal(lab.cpu().numpy()[clear], labr[clear])
+
+
+# --------------------------------------------------------------- priorities ---
+
+def _gpu_priorities(w, delta, alpha=None, with_entropy=True):
+    a = w.arrays
+    n = w.n
+    t = [dev(delta), dev(a["logp_target"]), dev(a["logp_behaviour"]), dev(a["entropy"]) if with_entropy else None]
+    mass = torch.empty(n, dtype=torch.float32, device="cuda")
+    q = torch.empty(n, dtype=torch.int32, device="cuda")
+    distrl.distrl_compute_priorities(t[0], t[1], t[2], t[3], prio_cfg_of(w, alpha), mass, q)
+    torch.cuda.synchronize()
+    return mass.cpu().numpy(), q.cpu().numpy().view(np.uint32)
+
+
+@pytest.mark.parametrize("index,alpha,with_entropy", [(0, 0.5, True), (0, 1.0, True), (1, 0.5, True), (1, 1.0, False),
+                                                      (1, 0.7, True), (2, 0.5, True), (3, 0.5, True)])
+def test_priorities(index, alpha, with_entropy):
+    w = synth.make_workload(index)
+    a = w.arrays
+    _, _, dl = oracle.retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"],
+                              w.gamma, w.lam)
+    delta = dl.astype(np.float32)
+    if w.heavy_tail:
+        delta = (delta * synth.heavy_tail_scale(w)).astype(np.float32)
+    mass, q = _gpu_priorities(w, delta, alpha, with_entropy)
+    ref = oracle.priority_mass(delta, a["logp_target"], a["logp_behaviour"], a["entropy"] if with_entropy else None,
+                               w.w_td, w.w_rho, w.w_ent, w.rho_clip, alpha)
+    assert_close(mass, ref, "prio_mass")
+    # integer stage: the device's q is exactly Q(device's fp32 mass)
+    np.testing.assert_array_equal(q, oracle.quantise(mass, w.scale))
+    assert q.min() >= 1
+    # informational: how often Q of the oracle's own mass differs
+    q_ref = oracle.quantise(ref.astype(np.float32), w.scale)
+    diff = np.abs(q.astype(np.int64) - q_ref.astype(np.int64))
+    assert np.all(diff <= np.maximum(1, 4e-7 * q_ref))
+
+
+def test_priority_quantiser_edges_on_device():
+    # drive the device quantiser through its corner cases with alpha = 1, w = (1, 0, 0): mass = |delta|
+    S = 2.0 ** 20
+    vals = np.array([0.0, 2.0 ** -21, 1.5 / S, 2.5 / S, 3.5 / S, 1.0, 4095.999, 4096.0, 1e30, np.inf, np.nan,
+                     -3.0, 2.0 ** -30], dtype=np.float32)
+    z = torch.zeros(vals.shape[0], dtype=torch.float32, device="cuda")
+    mass = torch.empty_like(z)
+    q = torch.empty(vals.shape[0], dtype=torch.int32, device="cuda")
+    distrl.distrl_compute_priorities(dev(vals), z, z, z, distrl.make_prio_cfg(1.0, 0.0, 0.0, 2.0, 1.0, S), mass, q)
+    got = q.cpu().numpy().view(np.uint32)
+    np.testing.assert_array_equal(got, oracle.quantise(mass.cpu().numpy(), S))
+    assert got[0] == 1 and got[2] == 2 and got[3] == 2 and got[4] == 4 and got[7] == 2 ** 32 - 1 and got[10] == 1
+
+
+def test_trajectory_level_priorities():
+    w = synth.make_workload(1)
+    a = w.arrays
+    off = np.sort(np.concatenate([a["traj_offsets"], a["traj_offsets"][[5, 5, 100]]]))   # add empty trajectories
+    _, _, dl = oracle.retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"],
+                              w.gamma, w.lam)
+    delta = dl.astype(np.float32)
+    m = off.shape[0] - 1
+    mass = torch.empty(m, dtype=torch.float32, device="cuda")
+    q = torch.empty(m, dtype=torch.int32, device="cuda")
+    distrl.distrl_compute_priorities_traj(dev(off), dev(delta), dev(a["logp_target"]), dev(a["logp_behaviour"]),
+                                          dev(a["entropy"]), prio_cfg_of(w), mass, q)
+    ref = oracle.priority_mass_traj(off, delta, a["logp_target"], a["logp_behaviour"], a["entropy"], w.w_td, w.w_rho,
+                                    w.w_ent, w.rho_clip, w.alpha)
+    assert_close(mass.cpu().numpy(), ref, "traj prio_mass")
+    np.testing.assert_array_equal(q.cpu().numpy().view(np.uint32), oracle.quantise(mass.cpu().numpy(), w.scale))
+
+
+# ------------------------------------------------------------------ sampler ---
+
+def _masses(n, seed, heavy=True):
+    rng = np.random.default_rng(seed)
+    if heavy:
+        x = np.exp(rng.normal(0, 3, n)) * 2 ** 18
+        return np.clip(np.rint(x), 1, 2 ** 32 - 1).astype(np.uint32)
+    return rng.integers(1, 2 ** 32, size=n, dtype=np.uint64).astype(np.uint32)
+
+
+def _build(q):
+    tq = dev(q.view(np.int32))
+    ws = distrl.alloc_workspace(distrl.distrl_sampler_workspace_bytes(q.shape[0]))
+    distrl.distrl_workspace_init(ws)
+    return distrl.distrl_build_sampler(tq, ws), tq, ws
+
+
+def _check_tree(s, q):
+    got, info = read_tree(s)
+    want = tree_from_q(q, info)
+    for l, (g, x) in enumerate(zip(got, want), start=1):
+        np.testing.assert_array_equal(g, x, err_msg="level %d" % l)
+    tot = torch.zeros(1, dtype=torch.int64, device="cuda")
+    distrl.distrl_sampler_total(s, tot)
+    _, total = oracle.prefix(q)
+    assert int(tot.cpu().numpy().view(np.uint64)[0]) == total
+    assert int(got[-1].sum(dtype=np.uint64)) == total
+
+
+def _sample(s, u, beta, normalise=True):
+    k = u.shape[0]
+    idx = torch.full((k,), -1, dtype=torch.int64, device="cuda")
+    wts = torch.full((k,), float("nan"), dtype=torch.float32, device="cuda")
+    distrl.distrl_sample(s, dev(u.view(np.int64)), beta, normalise, idx, wts)
+    torch.cuda.synchronize()
+    return idx.cpu().numpy(), wts.cpu().numpy()
+
+
+@pytest.mark.parametrize("n", [1, 2, 127, 128, 129, 4095, 4096, 4097, 131073, 1 << 20, (1 << 22) + 5])
+@pytest.mark.parametrize("heavy", [True, False])
+def test_sampler_build_and_sample(n, heavy):
+    q = _masses(n, n + int(heavy), heavy)
+    s, tq, ws = _build(q)
+    _check_tree(s, q)
+    rng = np.random.default_rng(n)
+    u = rng.integers(0, 1 << 64, size=513, dtype=np.uint64)
+    u[:4] = [0, 2 ** 64 - 1, 2 ** 63, 1]
+    idx, wts = _sample(s, u, 0.4)
+    np.testing.assert_array_equal(idx, sample_by_prefix(q, u))
+    sub = slice(0, 24 if n > 100000 else 513)
+    np.testing.assert_array_equal(idx[sub], oracle.sample_linear(q, u[sub]))       # the definition itself
+    assert_close(wts, oracle.is_weights(q, idx, 0.4, True), "is_weight")
+    assert wts.max() == 1.0
+    _, raw = _sample(s, u, 0.6, normalise=False)
+    assert_close(raw, oracle.is_weights(q, idx, 0.6, False), "is_weight raw")
+    assert distrl.distrl_get_status(ws) == 0
+    s.close()
+
+
+def test_sampling_brute_force_on_device():
+    # every threshold y in [0, total) must land on index i exactly q_i times
+    q = np.array([3, 1, 7, 1, 1, 12, 5] * 40, dtype=np.uint32)
+    total = int(q.sum())
+    u = np.array([-((-y * (1 << 64)) // total) for y in range(total)], dtype=np.uint64)
+    s, tq, ws = _build(q)
+    idx, _ = _sample(s, u, 0.4)
+    np.testing.assert_array_equal(np.bincount(idx, minlength=q.shape[0]), q)
+    s.close()
+
+
+def _update(s, w_cfg, idx, nd, lp, lm, ent):
+    k = idx.shape[0]
+    mass = torch.full((k,), float("nan"), dtype=torch.float32, device="cuda")
+    distrl.distrl_update_priorities(s, dev(idx), dev(nd), lp, lm, ent, w_cfg, mass)
+    torch.cuda.synchronize()
+    return mass.cpu().numpy()
+
+
+@pytest.mark.parametrize("index,k", [(0, 32), (1, 256), (1, 9000), (2, 1024), (2, 20000)])
+def test_update_equals_rebuild(index, k):
+    w = synth.make_workload(index)
+    a = w.arrays
+    cfg = prio_cfg_of(w)
+    _, _, dl = oracle.retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"],
+                              w.gamma, w.lam)
+    mass0 = oracle.priority_mass(dl, a["logp_target"], a["logp_behaviour"], a["entropy"], w.w_td, w.w_rho, w.w_ent,
+                                 w.rho_clip, w.alpha)
+    q = oracle.quantise(mass0.astype(np.float32), w.scale)
+    s, tq, ws = _build(q)
+    lp, lm, ent = dev(a["logp_target"]), dev(a["logp_behaviour"]), dev(a["entropy"])
+    for rnd in range(3):
+        u = synth.uniforms(w, rnd, k)
+        idx, wts = _sample(s, u, w.beta)
+        np.testing.assert_array_equal(idx, sample_by_prefix(q, u))
+        assert_close(wts, oracle.is_weights(q, idx, w.beta, True), "is_weight")
+        if rnd == 0:   # force duplicates, also across the chunk boundary of large batches
+            idx[k // 2:k // 2 + 5] = idx[0]
+            idx[-1] = idx[1]
+        nd = synth.fresh_abs_delta(w, rnd, k)
+        gmass = _update(s, cfg, idx, nd, lp, lm, ent)
+        q_ref = q.copy()
+        omass = oracle.update(q_ref, idx, nd, a["logp_target"], a["logp_behaviour"], a["entropy"], w.w_td, w.w_rho,
+                              w.w_ent, w.rho_clip, w.alpha, w.scale)
+        assert_close(gmass, omass, "update mass")
+        # integer stage: sequential requantisation of the device's own masses
+        oracle.update_from_mass(q, idx, gmass, w.scale)
+        np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), q)
+        assert np.all(np.abs(q.astype(np.int64) - q_ref.astype(np.int64)) <= np.maximum(1, 4e-7 * q_ref))
+        _check_tree(s, q)                      # incremental repair == rebuild from scratch
+    assert distrl.distrl_get_status(ws) == 0
+    s.close()
+
+
+def test_update_rejects_bad_index_but_applies_the_rest():
+    q = _masses(5000, 1)
+    s, tq, ws = _build(q)
+    z = torch.zeros(5000, dtype=torch.float32, device="cuda")
+    idx = np.array([7, 5000, -1, 9], dtype=np.int64)
+    nd = np.array([4.0, 1.0, 1.0, 9.0], dtype=np.float32)
+    _update(s, distrl.make_prio_cfg(1.0, 0.0, 0.0, 2.0, 0.5, 2.0 ** 20), idx, nd, z, z, z)
+    assert distrl.distrl_get_status(ws) == distrl.binding.ERR_INDEX
+    q[7] = 2 << 20
+    q[9] = 3 << 20
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), q)
+    _check_tree(s, q)
+    assert distrl.distrl_get_status(ws) == 0       # reading cleared it
+    s.close()
+
+
+def test_full_path_rounds_config3():
+    """Workload 3 end to end at full size in the call sequence the benchmark times."""
+    w = synth.make_workload(3)
+    a = w.arrays
+    n = w.n
+    out = check_retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"],
+                        w.gamma, w.lam)
+    delta = (out["td_delta"] * synth.heavy_tail_scale(w)).astype(np.float32)
+    cfg = prio_cfg_of(w)
+    lp, lm, ent = dev(a["logp_target"]), dev(a["logp_behaviour"]), dev(a["entropy"])
+    mass = torch.empty(n, dtype=torch.float32, device="cuda")
+    tq = torch.empty(n, dtype=torch.int32, device="cuda")
+    distrl.distrl_compute_priorities(dev(delta), lp, lm, ent, cfg, mass, tq)
+    q = oracle.quantise(mass.cpu().numpy(), w.scale)
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), q)
+    ws = distrl.alloc_workspace(distrl.distrl_sampler_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws)
+    s = distrl.distrl_build_sampler(tq, ws)
+    _check_tree(s, q)
+    for rnd in range(w.rounds):
+        u = synth.uniforms(w, rnd)
+        idx, wts = _sample(s, u, w.beta)
+        np.testing.assert_array_equal(idx, sample_by_prefix(q, u))
+        if rnd in (0, 57):
+            np.testing.assert_array_equal(idx[:6], oracle.sample_linear(q, u[:6]))
+        assert_close(wts, oracle.is_weights(q, idx, w.beta, True), "is_weight")
+        nd = synth.fresh_abs_delta(w, rnd)
+        gmass = _update(s, cfg, idx, nd, lp, lm, ent)
+        oracle.update_from_mass(q, idx, gmass, w.scale)
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), q)
+    _check_tree(s, q)
+    assert distrl.distrl_get_status(ws) == 0
+    s.close()
