@@ -356,3 +356,91 @@ def test_full_path_rounds_config3():
     _check_tree(s, q)
     assert distrl.distrl_get_status(ws) == 0
     s.close()
+
+
+# -------------------------------------------------------------- token level ---
+
+def _token_case(off, sto, tok_p, tok_m, seed, gamma=0.99, lam=0.95, **kw):
+    n = int(off[-1])
+    rng = np.random.default_rng(seed)
+    r = rng.normal(0, 1, n).astype(np.float32)
+    V = rng.random(n, dtype=np.float32)
+    lp = oracle.token_logp(sto, oracle.bf16_bits_to_f64(tok_p))
+    lm = oracle.token_logp(sto, oracle.bf16_bits_to_f64(tok_m))
+    out = gpu_retrace(off, r, V, None, None, gamma, lam, tokens=(sto, tok_p, tok_m), want_logp=True, **kw)
+    assert out["status"] == 0
+    vt, adv, dl = oracle.retrace(off, r, V, lp, lm, gamma, lam)
+    assert_close(out["logp_target"], lp, "token logp_target")
+    assert_close(out["logp_behaviour"], lm, "token logp_behaviour")
+    assert_close(out["v_target"], vt, "v_target")
+    assert_close(out["advantage"], adv, "advantage")
+    assert_close(out["td_delta"], dl, "td_delta")
+
+
+@pytest.mark.parametrize("n", [1000, 50000, 300001])
+def test_token_level_workload(n):
+    w = synth.make_workload(4, n_override=n)
+    a = w.arrays
+    _token_case(a["traj_offsets"], a["step_token_offsets"], a["tok_logp_target"], a["tok_logp_behaviour"], n,
+                w.gamma, w.lam)
+
+
+@pytest.mark.parametrize("counts", ["all32", "zeros_and_ones", "one_huge", "wide"])
+def test_token_level_count_extremes(counts):
+    # all32: every tile owns more tokens than one staging pass holds; zeros_and_ones: empty steps;
+    # one_huge: a single step with 70,000 tokens; wide: counts up to 200.
+    n = 5000
+    rng = np.random.default_rng(17)
+    cnt = {"all32": np.full(n, 32), "zeros_and_ones": rng.integers(0, 2, n),
+           "one_huge": np.where(np.arange(n) == 2500, 70000, 1), "wide": rng.integers(0, 201, n)}[counts]
+    sto = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int64)
+    nt = int(sto[-1])
+    shrink = np.float32(max(1, cnt.max() // 32))     # keep the per-step sums in a sane range
+    tok_m = synth.f32_to_bf16_bits((rng.standard_normal(nt) * 0.3 - 0.3).astype(np.float32) / shrink)
+    tok_p = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(tok_m) +
+                                   (rng.standard_normal(nt) * 0.05).astype(np.float32) / shrink)
+    off = synth.adversarial_offsets("long_mixed", n, tile=1024)
+    _token_case(off, sto, tok_p, tok_m, 3)
+
+
+def test_token_level_single_token_steps_equal_plain_logp():
+    # one token per step: the token path must agree with the fp32-logp path on the same numbers
+    n = 30000
+    rng = np.random.default_rng(21)
+    off = synth.adversarial_offsets("long_mixed", n)
+    tok_m = synth.f32_to_bf16_bits(rng.normal(-5, 2, n).astype(np.float32))
+    tok_p = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(tok_m) + rng.normal(0, 0.5, n).astype(np.float32))
+    sto = np.arange(n + 1, dtype=np.int64)
+    r = rng.normal(0, 1, n).astype(np.float32)
+    V = rng.random(n, dtype=np.float32)
+    a = gpu_retrace(off, r, V, None, None, 0.99, 0.95, tokens=(sto, tok_p, tok_m))
+    b = gpu_retrace(off, r, V, synth.bf16_bits_to_f32(tok_p), synth.bf16_bits_to_f32(tok_m), 0.99, 0.95)
+    for key in ("v_target", "advantage", "td_delta"):
+        assert_close(a[key], b[key].astype(np.float64), key, tol=1e-6)
+
+
+def test_token_level_unaligned_token_arrays():
+    w = synth.make_workload(4, n_override=20000)
+    a = w.arrays
+    sto, tp, tm = a["step_token_offsets"], a["tok_logp_target"], a["tok_logp_behaviour"]
+    n = w.n
+    rng = np.random.default_rng(2)
+    r = rng.normal(0, 1, n).astype(np.float32)
+    V = rng.random(n, dtype=np.float32)
+    t_off, t_r, t_V, t_sto = dev(a["traj_offsets"]), dev(r), dev(V), dev(sto)
+    bufp = torch.empty(tp.shape[0] + 1, dtype=torch.bfloat16, device="cuda")
+    bufm = torch.empty(tp.shape[0] + 1, dtype=torch.bfloat16, device="cuda")
+    bufp[1:].copy_(torch.from_numpy(tp).view(torch.bfloat16))
+    bufm[1:].copy_(torch.from_numpy(tm).view(torch.bfloat16))
+    batch = distrl.make_batch(t_off, t_r, t_V, None, None, None, t_sto, bufp[1:], bufm[1:])
+    vt = torch.empty(n, dtype=torch.float32, device="cuda")
+    adv = torch.empty(n, dtype=torch.float32, device="cuda")
+    ws = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws)
+    distrl.distrl_retrace_targets(batch, w.gamma, w.lam, vt, adv, workspace=ws)
+    assert distrl.distrl_get_status(ws) == 0
+    lp = oracle.token_logp(sto, oracle.bf16_bits_to_f64(tp))
+    lm = oracle.token_logp(sto, oracle.bf16_bits_to_f64(tm))
+    o_vt, o_adv, _ = oracle.retrace(a["traj_offsets"], r, V, lp, lm, w.gamma, w.lam)
+    assert_close(vt.cpu().numpy(), o_vt, "v_target")
+    assert_close(adv.cpu().numpy(), o_adv, "advantage")
