@@ -120,7 +120,8 @@ def _config(w, args, l2):
                         % (w.name, w.index, w.n, w.m, w.batch, w.rounds),
             "gamma": w.gamma, "lambda": w.lam, "alpha": w.alpha, "beta": w.beta, "fixed_point_scale": w.scale,
             "parallelism": "independent replay shard per GPU (no data-path collective)" if args.gpus > 1 else "1 GPU",
-            "l2": l2}
+            "l2": l2,
+            "rounds_launch": "eager" if getattr(args, "no_graph", False) else "caller-side CUDA graph of the rounds"}
 
 
 # --------------------------------------------------------------------------- CUDA legs
@@ -230,7 +231,27 @@ def run_ours(args):
     torch.cuda.synchronize()
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    launches_per_step = 2 + 1 + 2 + 2 * R
+    launches_per_step = 2 + 1 + 2 + 3 * R   # scan prep + scan, priorities, 2 build, (sample, claim, apply) x R
+
+    def rounds(s):
+        for r in range(R):
+            distrl.distrl_sample(s, d_u[r], w.beta, True, idx[r], wts[r])
+            distrl.distrl_update_priorities(s, idx[r], d_nd[r], dv["logp_target"], dv["logp_behaviour"],
+                                            dv["entropy"], cfg, None)
+
+    # The R sample->refresh rounds are launch-bound (3 short kernels each), so the caller records them once
+    # into a CUDA graph and replays it every step.  The sampler handle only holds pointers into ws_s and q,
+    # which never move, so the recorded launches stay valid when the tree is rebuilt each step.
+    graph = None
+    s_graph = None
+    if not args.no_graph:
+        s_graph = distrl.distrl_build_sampler(q, ws_s)
+        rounds(s_graph)                       # first use outside capture (one-time function attributes)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            rounds(s_graph)
+        torch.cuda.synchronize()
 
     def step(marks=None):
         if marks: marks[0].record()
@@ -240,10 +261,10 @@ def run_ours(args):
         if marks: marks[2].record()
         s = distrl.distrl_build_sampler(q, ws_s)
         if marks: marks[3].record()
-        for r in range(R):
-            distrl.distrl_sample(s, d_u[r], w.beta, True, idx[r], wts[r])
-            distrl.distrl_update_priorities(s, idx[r], d_nd[r], dv["logp_target"], dv["logp_behaviour"],
-                                            dv["entropy"], cfg, None)
+        if graph is not None:
+            graph.replay()
+        else:
+            rounds(s)
         if marks: marks[4].record()
         s.close()
 
@@ -366,6 +387,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=sorted(WORKLOAD_INDEX), default="large")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch the sampling rounds one call at a time")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -9,11 +9,11 @@
 //   build  : one streaming pass over q writes levels 1 and 2, one small block
 //            finishes the levels above;
 //   sample : one warp per draw; per level one coalesced 256-byte load, a
-//            shuffle prefix sum and a ballot;
-//   update : one block; a shared-memory hash table elects, for every distinct
-//            index, the highest batch position (what a sequential loop would
-//            leave), the winners store the new mass and add new - old to every
-//            ancestor, so the tree stays bit-identical to a rebuild.
+//            shuffle prefix sum and a ballot; the top levels sit in shared memory;
+//   update : a claim word per transition elects, for every distinct index, the
+//            highest batch position (what a sequential loop would leave); the
+//            winners store the new mass and add new - old to every ancestor, so
+//            the tree stays bit-identical to a rebuild.
 #include "priority.cuh"
 
 #include <new>
@@ -23,12 +23,11 @@ namespace distrl {
 constexpr int kLeaf = 128;      // masses per level-1 entry
 constexpr int kFan = 32;        // fan-out above level 1
 constexpr int kMaxLevels = 8;   // enough for n <= 2^33
-constexpr int kSampleThreads = 256;
-constexpr int kUpdateThreads = 1024;
-constexpr int kUpdateChunk = 8192;              // batch positions per update launch
-constexpr int kHashSlots = 2 * kUpdateChunk;    // load factor <= 0.5
-constexpr int kPosBits = 13;                    // log2(kUpdateChunk)
-constexpr int kAccCap = 2048;                   // tree entries accumulated in shared memory
+constexpr int kSampleThreads = 512;
+constexpr int kTopCap = 4352;                   // tree entries a sampling block caches in shared memory
+constexpr int kUpdateThreads = 256;
+constexpr int kUpdateChunk = 65536;             // batch positions per pair of update launches
+constexpr int kAccCap = 640;                    // tree entries an update block accumulates in shared memory
 
 struct Tree {
     int levels;                     // sum levels 1..levels
@@ -39,7 +38,8 @@ struct Tree {
     WorkspaceHeader *hdr;
 };
 
-static size_t tree_layout(int64_t n, void *base, Tree *t, size_t *offsets) {
+static size_t tree_layout(int64_t n, void *base, Tree *t, size_t *offsets, size_t *claim_off = nullptr,
+                          size_t *newq_off = nullptr) {
     int64_t count[kMaxLevels + 1] = {0};
     int levels = 1;
     count[1] = n > 0 ? ceil_div(n, kLeaf) : 1;
@@ -53,6 +53,10 @@ static size_t tree_layout(int64_t n, void *base, Tree *t, size_t *offsets) {
         if (t) t->lvl[l] = reinterpret_cast<unsigned long long *>(static_cast<char *>(base) + o);
         o = round_up(o + sizeof(unsigned long long) * count[l], 256);
     }
+    if (claim_off) *claim_off = o;
+    o = round_up(o + sizeof(unsigned int) * (size_t)(n > 0 ? n : 1), 256);      // claim[n]
+    if (newq_off) *newq_off = o;
+    o = round_up(o + sizeof(uint32_t) * (size_t)kUpdateChunk, 256);             // newq[kUpdateChunk]
     if (t) {
         t->levels = levels;
         t->n = n;
@@ -146,7 +150,9 @@ __global__ void total_kernel(Tree t, unsigned long long *out) {
 }
 
 // ---------------------------------------------------------------------------
-// sample: one warp per draw.
+// sample: one warp per draw.  The small top levels of the tree are copied into
+// shared memory once per block, so a draw pays one global round trip for that
+// copy plus one per remaining level and one for the leaf group.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ int pick_lane(unsigned long long incl, unsigned long long v, unsigned long long y) {
     unsigned int mask = __ballot_sync(0xffffffffu, incl > y);
@@ -156,16 +162,27 @@ __device__ __forceinline__ int pick_lane(unsigned long long incl, unsigned long 
     return nz ? (31 - __clz(nz)) : 0;
 }
 
+struct TopCache {
+    int from;                    // levels >= from are cached (levels + 1: none)
+    int off[kMaxLevels + 2];     // start of each cached level inside the cache
+    int total;                   // cached entries
+};
+
 __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
-    Tree t, const unsigned long long *__restrict__ u, int64_t k, float beta, int normalise,
+    Tree t, TopCache tc, const unsigned long long *__restrict__ u, int64_t k, float beta, int normalise,
     int64_t *__restrict__ idx_out, float *__restrict__ w_out, int vec_ok) {
+    __shared__ unsigned long long s_top[kTopCap];
     __shared__ int s_last;
     const int lane = threadIdx.x & 31;
+    for (int l = tc.from; l <= t.levels; ++l)
+        for (int i = threadIdx.x; i < t.count[l]; i += blockDim.x) s_top[tc.off[l] + i] = __ldcg(&t.lvl[l][i]);
+    __syncthreads();
     const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (j < k) {
         // top level: its entries sum to the total mass
         int l = t.levels;
-        unsigned long long v = (lane < t.count[l]) ? __ldcg(&t.lvl[l][lane]) : 0ull;
+        unsigned long long v = 0ull;
+        if (lane < t.count[l]) v = (l >= tc.from) ? s_top[tc.off[l] + lane] : __ldcg(&t.lvl[l][lane]);
         unsigned long long incl = warp_incl_scan_u64(v, lane);
         const unsigned long long total = __shfl_sync(0xffffffffu, incl, 31);
         unsigned long long y = __umul64hi(u[j], total);
@@ -176,7 +193,8 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
             node = node * kFan + c;
             if (--l == 0) break;
             int64_t i = node * kFan + lane;
-            v = (i < t.count[l]) ? __ldcg(&t.lvl[l][i]) : 0ull;
+            if (i < t.count[l]) v = (l >= tc.from) ? s_top[tc.off[l] + (int)i] : __ldcg(&t.lvl[l][i]);
+            else v = 0ull;
             incl = warp_incl_scan_u64(v, lane);
         }
         // leaf group `node`: 128 masses, 4 per lane
@@ -197,12 +215,16 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
             int e = 0;
             while (e < 3 && y >= qv[e]) { y -= qv[e]; ++e; }
             int64_t idx = p + e;
-            if (idx >= t.n) { idx = t.n - 1; set_status(&t.hdr->status, DISTRL_ERR_INDEX); }
+            uint32_t qs = qv[e];
+            if (idx >= t.n) { idx = t.n - 1; qs = 1u; set_status(&t.hdr->status, DISTRL_ERR_INDEX); }
             idx_out[j] = idx;
             if (w_out) {
-                uint32_t qs = qv[e];
-                if (normalise) atomicMin(&t.hdr->qmin, qs);
-                else w_out[j] = powf((float)((double)t.n * (double)qs / (double)total), -beta);
+                if (normalise) {
+                    atomicMin(&t.hdr->qmin, qs);
+                    w_out[j] = __uint_as_float(qs); // parked here until the batch minimum is known
+                } else {
+                    w_out[j] = powf((float)((double)t.n * (double)qs / (double)total), -beta);
+                }
             }
         }
     }
@@ -218,10 +240,10 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    const unsigned int qmin = atomicMin(&t.hdr->qmin, 0xffffffffu); // atomic read
+    const double qmin = (double)atomicMin(&t.hdr->qmin, 0xffffffffu); // atomic read
     for (int64_t i = threadIdx.x; i < k; i += blockDim.x) {
-        uint32_t qs = __ldcg(t.q + __ldcg(idx_out + i));
-        w_out[i] = powf((float)((double)qs / (double)qmin), -beta);
+        uint32_t qs = __float_as_uint(__ldcg(w_out + i));
+        w_out[i] = powf((float)((double)qs / qmin), -beta);
     }
     __syncthreads();
     if (threadIdx.x == 0) { // ready for the next call
@@ -231,87 +253,96 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
 }
 
 // ---------------------------------------------------------------------------
-// update: one block per chunk of <= kUpdateChunk batch positions.
+// update, in two launches per chunk of batch positions.
+//
+// A sequential loop over the batch leaves, for an index that occurs several
+// times, the value of its highest position.  claim[] has one word per
+// transition; position j competes for claim[idx[j]] and the highest one stays.
+// The table is never cleared: an entry c counts only if it names a position of
+// THIS batch that holds the same index (c < k and idx[c] == i), so whatever an
+// earlier call or uninitialised memory left behind is either ignored or is
+// itself a correct claim.
+//   claim kernel : gathers rho and H, computes the new mass and its fixed-point
+//                  image, competes for the claim;
+//   apply kernel : the winners store the new mass and add (new - old) to every
+//                  ancestor, so the tree equals a rebuild bit for bit.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ unsigned int hash_idx(unsigned long long key) {
-    key ^= key >> 33;
-    key *= 0xff51afd7ed558ccdull;
-    key ^= key >> 29;
-    return (unsigned int)key & (kHashSlots - 1);
-}
+struct UpdateWs {
+    unsigned int *claim; // [n]
+    uint32_t *newq;      // [kUpdateChunk]
+};
 
-__global__ void __launch_bounds__(kUpdateThreads) update_kernel(
-    Tree t, const int64_t *__restrict__ idx, int k, const float *__restrict__ new_abs_delta,
+__global__ void __launch_bounds__(kUpdateThreads) update_claim_kernel(
+    Tree t, UpdateWs uw, const int64_t *__restrict__ idx, int k, const float *__restrict__ new_abs_delta,
     const float *__restrict__ lp, const float *__restrict__ lm, const float *__restrict__ ent, PrioCfg c,
     float *__restrict__ mass_out) {
-    extern __shared__ unsigned long long s_mem[];
-    unsigned long long *s_tab = s_mem;             // [kHashSlots] (index + 1) << kPosBits | position
-    unsigned long long *s_acc = s_mem + kHashSlots; // [kAccCap] pending sums for the small top levels
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= k) return;
+    const int64_t i = idx[j];
+    if (i < 0 || i >= t.n) {
+        set_status(&t.hdr->status, DISTRL_ERR_INDEX);
+        if (mass_out) mass_out[j] = 0.f;
+        return;
+    }
+    const float p = __ldg(lp + i), m = __ldg(lm + i);
+    const float h = ent ? __ldg(ent + i) : -p;
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(t.q + i)); // the apply kernel reads it next
+    unsigned int *slot = uw.claim + i;
+    unsigned int old = *reinterpret_cast<volatile unsigned int *>(slot);
+    while (true) {
+        const bool legit = old < (unsigned int)k && idx[old] == i;
+        if (legit && old >= (unsigned int)j) break;
+        const unsigned int prev = atomicCAS(slot, old, (unsigned int)j);
+        if (prev == old) break;
+        old = prev;
+    }
+    const float mass = prio_mass(new_abs_delta[j], p, m, h, c);
+    if (mass_out) mass_out[j] = mass;
+    uw.newq[j] = prio_quantise(mass, c.scale);
+}
 
-    // which levels accumulate in shared memory (from the top down, while they fit)
-    int acc_from = t.levels + 1; // levels >= acc_from live in s_acc
-    int acc_off[kMaxLevels + 2];
-    {
-        int used = 0;
+__global__ void __launch_bounds__(kUpdateThreads) update_apply_kernel(Tree t, UpdateWs uw,
+                                                                      const int64_t *__restrict__ idx, int k) {
+    __shared__ unsigned long long s_acc[kAccCap]; // pending sums of the small top levels, per block
+    __shared__ int s_acc_off[kMaxLevels + 2];
+    __shared__ int s_acc_from, s_acc_used;
+    if (threadIdx.x == 0) {
+        int used = 0, from = t.levels + 1;
         for (int l = t.levels; l >= 1; --l) {
             if (used + t.count[l] > kAccCap) break;
-            acc_off[l] = used;
+            s_acc_off[l] = used;
             used += (int)t.count[l];
-            acc_from = l;
+            from = l;
         }
-        for (int i = threadIdx.x; i < used; i += blockDim.x) s_acc[i] = 0ull;
+        s_acc_from = from;
+        s_acc_used = used;
     }
-    for (int i = threadIdx.x; i < kHashSlots; i += blockDim.x) s_tab[i] = 0ull;
     __syncthreads();
-
-    // phase 1: per distinct index keep the highest batch position
-    for (int j = threadIdx.x; j < k; j += blockDim.x) {
-        int64_t i = idx[j];
-        if (i < 0 || i >= t.n) { set_status(&t.hdr->status, DISTRL_ERR_INDEX); continue; }
-        const unsigned long long tag = (unsigned long long)(i + 1);
-        const unsigned long long packed = (tag << kPosBits) | (unsigned long long)j;
-        unsigned int h = hash_idx(tag);
-        while (true) {
-            unsigned long long cur = s_tab[h];
-            if (cur == 0ull) {
-                cur = atomicCAS(&s_tab[h], 0ull, packed);
-                if (cur == 0ull) break;
+    const int acc_from = s_acc_from, used = s_acc_used;
+    for (int i = threadIdx.x; i < used; i += blockDim.x) s_acc[i] = 0ull;
+    __syncthreads();
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < k) {
+        const int64_t i = idx[j];
+        if (i >= 0 && i < t.n && __ldcg(uw.claim + i) == (unsigned int)j) {
+            const uint32_t qn = uw.newq[j], qo = __ldcg(t.q + i);
+            if (qn != qo) {
+                t.q[i] = qn;
+                const unsigned long long diff = (unsigned long long)qn - (unsigned long long)qo; // mod 2^64
+                int64_t node = i / kLeaf;
+                for (int l = 1; l <= t.levels; ++l) {
+                    if (l >= acc_from) atomicAdd(&s_acc[s_acc_off[l] + (int)node], diff);
+                    else atomicAdd(&t.lvl[l][node], diff);
+                    node /= kFan;
+                }
             }
-            if ((cur >> kPosBits) == tag) { atomicMax(&s_tab[h], packed); break; }
-            h = (h + 1) & (kHashSlots - 1);
         }
     }
     __syncthreads();
-
-    // phase 2: every position computes its mass; the winner applies it
-    for (int j = threadIdx.x; j < k; j += blockDim.x) {
-        int64_t i = idx[j];
-        if (i < 0 || i >= t.n) { if (mass_out) mass_out[j] = 0.f; continue; }
-        float p = lp[i];
-        float mass = prio_mass(new_abs_delta[j], p, lm[i], ent ? ent[i] : -p, c);
-        if (mass_out) mass_out[j] = mass;
-        const unsigned long long tag = (unsigned long long)(i + 1);
-        unsigned int h = hash_idx(tag);
-        unsigned long long cur;
-        while (((cur = s_tab[h]) >> kPosBits) != tag) h = (h + 1) & (kHashSlots - 1);
-        if ((int)(cur & ((1u << kPosBits) - 1u)) != j) continue;
-        const uint32_t qn = prio_quantise(mass, c.scale), qo = t.q[i];
-        if (qn == qo) continue;
-        t.q[i] = qn;
-        const unsigned long long diff = (unsigned long long)qn - (unsigned long long)qo; // mod 2^64
-        int64_t node = i / kLeaf;
-        for (int l = 1; l <= t.levels; ++l) {
-            if (l >= acc_from) atomicAdd(&s_acc[acc_off[l] + (int)node], diff);
-            else atomicAdd(&t.lvl[l][node], diff);
-            node /= kFan;
-        }
-    }
-    __syncthreads();
-    // flush the shared-memory sums: this block is the only writer
     for (int l = acc_from; l <= t.levels; ++l)
         for (int i = threadIdx.x; i < t.count[l]; i += blockDim.x) {
-            unsigned long long d = s_acc[acc_off[l] + i];
-            if (d) t.lvl[l][i] += d;
+            unsigned long long d = s_acc[s_acc_off[l] + i];
+            if (d) atomicAdd(&t.lvl[l][i], d);
         }
 }
 
@@ -321,6 +352,8 @@ using namespace distrl;
 
 struct distrl_sampler {
     Tree tree;
+    TopCache top;
+    UpdateWs upd;
     size_t offsets[kMaxLevels + 1];
     int vec_ok;
 };
@@ -341,7 +374,21 @@ extern "C" int distrl_build_sampler(uint32_t *prio_q, int64_t n, void *workspace
         return DISTRL_ERR_WORKSPACE;
     distrl_sampler *s = new (std::nothrow) distrl_sampler();
     if (!s) return DISTRL_ERR_CUDA;
-    tree_layout(n, workspace, &s->tree, s->offsets);
+    size_t claim_off = 0, newq_off = 0;
+    tree_layout(n, workspace, &s->tree, s->offsets, &claim_off, &newq_off);
+    s->upd.claim = reinterpret_cast<unsigned int *>(static_cast<char *>(workspace) + claim_off);
+    s->upd.newq = reinterpret_cast<uint32_t *>(static_cast<char *>(workspace) + newq_off);
+    {   // which top levels fit the sampling blocks' shared-memory cache
+        TopCache &tc = s->top;
+        tc.from = s->tree.levels + 1;
+        tc.total = 0;
+        for (int l = s->tree.levels; l >= 1; --l) {
+            if (tc.total + s->tree.count[l] > kTopCap) break;
+            tc.off[l] = tc.total;
+            tc.total += (int)s->tree.count[l];
+            tc.from = l;
+        }
+    }
     s->tree.q = prio_q;
     s->vec_ok = aligned_to(prio_q, 16) ? 1 : 0;
     *out = s;
@@ -369,7 +416,7 @@ extern "C" int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k
     if (!aligned_to(u_fix, 8) || !aligned_to(idx_out, 8) || !aligned_to(is_weight_out, 4)) return DISTRL_ERR_ALIGN;
     const int64_t blocks = ceil_div(k * 32, kSampleThreads);
     sample_kernel<<<(unsigned)blocks, kSampleThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        s->tree, reinterpret_cast<const unsigned long long *>(u_fix), k, beta, normalise, idx_out, is_weight_out,
+        s->tree, s->top, reinterpret_cast<const unsigned long long *>(u_fix), k, beta, normalise, idx_out, is_weight_out,
         s->vec_ok);
     DISTRL_CUDA_TRY(cudaGetLastError());
     return DISTRL_OK;
@@ -389,22 +436,15 @@ extern "C" int distrl_update_priorities(distrl_sampler *s, const int64_t *idx, i
     if (!aligned_to(idx, 8) || !aligned_to(new_abs_delta, 4) || !aligned_to(lp, 4) || !aligned_to(lm, 4) ||
         !aligned_to(entropy, 4) || !aligned_to(mass_out, 4))
         return DISTRL_ERR_ALIGN;
-    const size_t smem = sizeof(unsigned long long) * (kHashSlots + kAccCap);
-    {   // opt in to the large dynamic shared-memory window, once per device
-        static bool attr_set[64] = {false};
-        int dev = 0;
-        DISTRL_CUDA_TRY(cudaGetDevice(&dev));
-        if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-            DISTRL_CUDA_TRY(cudaFuncSetAttribute(update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            if (dev >= 0 && dev < 64) attr_set[dev] = true;
-        }
-    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // chunks run one after another on the stream, so "later position wins" also holds across chunks
     for (int64_t o = 0; o < k; o += kUpdateChunk) {
-        int kc = (int)((k - o < kUpdateChunk) ? (k - o) : kUpdateChunk);
-        update_kernel<<<1, kUpdateThreads, smem, st>>>(s->tree, idx + o, kc, new_abs_delta + o, lp, lm, entropy, c,
-                                                       mass_out ? mass_out + o : nullptr);
+        const int kc = (int)((k - o < kUpdateChunk) ? (k - o) : kUpdateChunk);
+        const unsigned grid = (unsigned)ceil_div(kc, kUpdateThreads);
+        update_claim_kernel<<<grid, kUpdateThreads, 0, st>>>(s->tree, s->upd, idx + o, kc, new_abs_delta + o, lp, lm,
+                                                            entropy, c, mass_out ? mass_out + o : nullptr);
+        DISTRL_CUDA_TRY(cudaGetLastError());
+        update_apply_kernel<<<grid, kUpdateThreads, 0, st>>>(s->tree, s->upd, idx + o, kc);
         DISTRL_CUDA_TRY(cudaGetLastError());
     }
     return DISTRL_OK;

@@ -47,8 +47,10 @@ def test_workspace_sizes_grow_and_are_aligned():
         assert a % 256 == 0 and b % 256 == 0 and a >= 256 and b >= 256
         assert a + b >= prev
         prev = a + b
-    # the tree of 2^24 masses: 131072 + 4096 + 128 + 4 uint64 entries
-    assert distrl.distrl_sampler_workspace_bytes(1 << 24) == 256 + 8 * (131072 + 4096 + 128) + 256
+    # 2^24 masses: header, tree levels of 131072 + 4096 + 128 + 4 uint64 entries, one claim word per
+    # mass, and the 65536-entry staging array of the refresh
+    assert distrl.distrl_sampler_workspace_bytes(1 << 24) == \
+        256 + 8 * (131072 + 4096 + 128) + 256 + 4 * (1 << 24) + 4 * 65536
 
 
 def test_argument_validation_happens_before_any_device_work():
