@@ -110,6 +110,33 @@ int distrl_retrace_targets(const distrl_batch *batch, float gamma, float lambda,
                            void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * distrl_retrace_targets without a workspace argument.  (The paper has no
+ * counterpart: this is a convenience of this library.)
+ *
+ * Meant for callers that cannot allocate device memory when they need the
+ * targets -- for instance a learner whose framework has already reserved the
+ * whole GPU for its own pool, so that a further cudaMalloc fails or shrinks
+ * that pool, or a step loop that must stay clear of cudaMalloc because it
+ * stalls the whole device.  The scan's tile bookkeeping lives in a fixed
+ * array inside the library image (about 100 KB, held by every GPU that loads
+ * the library until the process exits), which limits the size:
+ *   n_transitions <= DISTRL_STATIC_MAX_N, else DISTRL_ERR_SIZE.
+ * Arguments and results are those of distrl_retrace_targets, plus
+ *   status_out_device : device int or NULL; receives the device status word of
+ *       this call (DISTRL_OK, DISTRL_ERR_OFFSETS, DISTRL_ERR_TIMEOUT).
+ * The call allocates nothing (no cudaMalloc / cudaFree, no library allocator).
+ * The first call on each device looks up the array's device address; make that
+ * first call outside any stream capture.  All calls on a device share the one
+ * array: issue them on one stream, or otherwise make sure two of them never
+ * run on the GPU at the same time -- overlapping calls race on it.
+ */
+#define DISTRL_STATIC_MAX_N ((int64_t)1 << 22)
+int distrl_retrace_targets_static(const distrl_batch *batch, float gamma, float lambda,
+                                  float *v_target, float *advantage, float *td_delta,
+                                  float *logp_target_out, float *logp_behaviour_out,
+                                  int *status_out_device, void *stream);
+
+/*
  * Monte-Carlo return of Section 5.1, G_t = sum_{k>=t} gamma^(k-t) r_k per
  * trajectory, and the label I[G_t > 0] the state-value classifier is trained
  * on.  Same scan as above with coefficient gamma and increment r_t.

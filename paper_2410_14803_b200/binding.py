@@ -69,6 +69,7 @@ def _load():
         "distrl_retrace_workspace_bytes": (sz, [i64]),
         "distrl_workspace_init": (ci, [vp, sz, vp]),
         "distrl_retrace_targets": (ci, [ctypes.POINTER(distrl_batch), f32, f32, vp, vp, vp, vp, vp, vp, sz, vp]),
+        "distrl_retrace_targets_static": (ci, [ctypes.POINTER(distrl_batch), f32, f32, vp, vp, vp, vp, vp, vp, vp]),
         "distrl_mc_returns": (ci, [ctypes.POINTER(distrl_batch), f32, vp, vp, vp, sz, vp]),
         "distrl_compute_priorities": (ci, [i64, vp, vp, vp, vp, ctypes.POINTER(distrl_prio_cfg), vp, vp, vp]),
         "distrl_compute_priorities_traj": (ci, [i64, i64, vp, vp, vp, vp, vp, ctypes.POINTER(distrl_prio_cfg),
@@ -168,6 +169,23 @@ def distrl_retrace_targets(batch: distrl_batch, gamma: float, lam: float, v_targ
         _ptr(td_delta, torch.float32), _ptr(logp_target_out, torch.float32),
         _ptr(logp_behaviour_out, torch.float32), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _stream(stream)), "distrl_retrace_targets")
+
+
+STATIC_MAX_N = 1 << 22
+
+
+def distrl_retrace_targets_static(batch: distrl_batch, gamma: float, lam: float, v_target, advantage, td_delta=None,
+                                  logp_target_out=None, logp_behaviour_out=None, status_out=None, stream=None):
+    """distrl_retrace_targets for callers that cannot allocate a workspace (N <= STATIC_MAX_N).
+
+    The tile bookkeeping sits in a fixed array inside the library, shared by every call on the
+    device: keep such calls on one stream.  `status_out` is an optional int32 CUDA tensor (1 element)
+    that receives the device status word of this call."""
+    _check(_load().distrl_retrace_targets_static(
+        ctypes.byref(batch), gamma, lam, _ptr(v_target, torch.float32), _ptr(advantage, torch.float32),
+        _ptr(td_delta, torch.float32), _ptr(logp_target_out, torch.float32),
+        _ptr(logp_behaviour_out, torch.float32), _ptr(status_out, torch.int32), _stream(stream)),
+        "distrl_retrace_targets_static")
 
 
 def distrl_mc_returns(batch: distrl_batch, gamma: float, mc_return=None, label=None, *, workspace, stream=None):
