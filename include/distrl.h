@@ -78,9 +78,10 @@ typedef struct {
 /* Bytes of workspace distrl_retrace_targets needs for N transitions (any M). */
 size_t distrl_retrace_workspace_bytes(int64_t n_transitions);
 
-/* Zero a workspace's status word.  Call once after allocating a workspace
- * (retrace or sampler) and before its first use; the status word is sticky
- * until distrl_get_status() reads it. */
+/* Zero-fill a workspace (retrace or sampler).  Call once after allocating it
+ * and before its first use: the status word at its start is sticky until
+ * distrl_get_status() reads it.  Everything else in a workspace is scratch
+ * that each call rewrites. */
 int distrl_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
 
 /*
@@ -118,7 +119,7 @@ int distrl_retrace_targets(const distrl_batch *batch, float gamma, float lambda,
  * whole GPU for its own pool, so that a further cudaMalloc fails or shrinks
  * that pool, or a step loop that must stay clear of cudaMalloc because it
  * stalls the whole device.  The scan's tile bookkeeping lives in a fixed
- * array inside the library image (about 100 KB, held by every GPU that loads
+ * array inside the library image (about 0.6 MB, held by every GPU that loads
  * the library until the process exits), which limits the size:
  *   n_transitions <= DISTRL_STATIC_MAX_N, else DISTRL_ERR_SIZE.
  * Arguments and results are those of distrl_retrace_targets, plus

@@ -20,7 +20,7 @@ using namespace distrl;
 extern "C" int distrl_workspace_init(void *workspace, size_t workspace_bytes, void *stream) {
     if (!workspace) return DISTRL_ERR_NULL;
     if (!aligned_to(workspace, 256) || workspace_bytes < kHeaderBytes) return DISTRL_ERR_WORKSPACE;
-    DISTRL_CUDA_TRY(cudaMemsetAsync(workspace, 0, kHeaderBytes, static_cast<cudaStream_t>(stream)));
+    DISTRL_CUDA_TRY(cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)));
     return DISTRL_OK;
 }
 

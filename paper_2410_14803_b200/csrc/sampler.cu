@@ -174,10 +174,13 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     __shared__ unsigned long long s_top[kTopCap];
     __shared__ int s_last;
     const int lane = threadIdx.x & 31;
-    for (int l = tc.from; l <= t.levels; ++l)
-        for (int i = threadIdx.x; i < t.count[l]; i += blockDim.x) s_top[tc.off[l] + i] = __ldcg(&t.lvl[l][i]);
-    __syncthreads();
     const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const unsigned long long uj = (j < k) ? __ldg(u + j) : 0ull; // in flight while the cache fills
+    for (int l = tc.from; l <= t.levels; ++l) {
+#pragma unroll 4
+        for (int i = threadIdx.x; i < t.count[l]; i += blockDim.x) s_top[tc.off[l] + i] = __ldcg(&t.lvl[l][i]);
+    }
+    __syncthreads();
     if (j < k) {
         // top level: its entries sum to the total mass
         int l = t.levels;
@@ -185,7 +188,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
         if (lane < t.count[l]) v = (l >= tc.from) ? s_top[tc.off[l] + lane] : __ldcg(&t.lvl[l][lane]);
         unsigned long long incl = warp_incl_scan_u64(v, lane);
         const unsigned long long total = __shfl_sync(0xffffffffu, incl, 31);
-        unsigned long long y = __umul64hi(u[j], total);
+        unsigned long long y = __umul64hi(uj, total);
         int64_t node = 0;
         while (true) {
             int c = pick_lane(incl, v, y);
@@ -241,9 +244,18 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     if (!s_last) return;
     __threadfence();
     const double qmin = (double)atomicMin(&t.hdr->qmin, 0xffffffffu); // atomic read
-    for (int64_t i = threadIdx.x; i < k; i += blockDim.x) {
-        uint32_t qs = __float_as_uint(__ldcg(w_out + i));
-        w_out[i] = powf((float)((double)qs / qmin), -beta);
+    for (int64_t i0 = threadIdx.x; i0 < k; i0 += 4 * (int64_t)blockDim.x) { // four loads in flight per thread
+        uint32_t qs[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int64_t i = i0 + e * (int64_t)blockDim.x;
+            qs[e] = (i < k) ? __float_as_uint(__ldcg(w_out + i)) : 1u;
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int64_t i = i0 + e * (int64_t)blockDim.x;
+            if (i < k) w_out[i] = powf((float)((double)qs[e] / qmin), -beta);
+        }
     }
     __syncthreads();
     if (threadIdx.x == 0) { // ready for the next call
