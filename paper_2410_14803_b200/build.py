@@ -29,6 +29,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC, "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("DISTRL_NVCC_EXTRA", "").split()   # e.g. -D overrides of tuning constants
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB_PATH)

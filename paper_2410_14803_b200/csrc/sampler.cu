@@ -173,7 +173,9 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     int64_t *__restrict__ idx_out, float *__restrict__ w_out, int vec_ok) {
     __shared__ unsigned long long s_top[kTopCap];
     __shared__ int s_last;
+    __shared__ unsigned int s_qmin; // smallest mass drawn by this block
     const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) s_qmin = 0xffffffffu;
     const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const unsigned long long uj = (j < k) ? __ldg(u + j) : 0ull; // in flight while the cache fills
     for (int l = tc.from; l <= t.levels; ++l) {
@@ -223,7 +225,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
             idx_out[j] = idx;
             if (w_out) {
                 if (normalise) {
-                    atomicMin(&t.hdr->qmin, qs);
+                    atomicMin(&s_qmin, qs);          // one global atomic per block, below
                     w_out[j] = __uint_as_float(qs); // parked here until the batch minimum is known
                 } else {
                     w_out[j] = powf((float)((double)t.n * (double)qs / (double)total), -beta);
@@ -236,6 +238,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     // weight belongs to the smallest sampled mass, so w_j = (q_j / q_min)^-beta.
     __syncthreads();
     if (threadIdx.x == 0) {
+        atomicMin(&t.hdr->qmin, s_qmin);
         __threadfence();
         unsigned int done = atomicAdd(&t.hdr->done, 1u);
         s_last = (done == gridDim.x - 1);
