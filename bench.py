@@ -195,7 +195,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    w = synth.make_workload(WORKLOAD_INDEX[args.workload])
+    w = synth.make_workload(WORKLOAD_INDEX[args.workload], shard=rank)   # every rank owns its own shard
     if w.token_level:
         raise SystemExit("token-level workload: use tests; bench times the fp32 workloads")
     a = w.arrays
@@ -328,10 +328,8 @@ def run_ours(args):
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     ms_per_step = total_ms / args.steps
-    if world > 1:
-        t = torch.tensor([ms_per_step, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step, e2e_ms = float(t[0]), float(t[1])
+    from paper_2410_14803_b200.shard import max_over_ranks
+    ms_per_step, e2e_ms = max_over_ranks([ms_per_step, e2e_ms], device="cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()

@@ -66,6 +66,25 @@ static size_t tree_layout(int64_t n, void *base, Tree *t, size_t *offsets, size_
     return o;
 }
 
+// mbarrier + 1-D bulk copy (global -> shared), used to fill the sampling blocks' cache
+__device__ __forceinline__ unsigned int smem_addr(const void *p) { return (unsigned int)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, unsigned int bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, unsigned int parity) {
+    unsigned int ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned int bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
 __device__ __forceinline__ unsigned long long warp_incl_scan_u64(unsigned long long v, int lane) {
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -171,18 +190,35 @@ struct TopCache {
 __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     Tree t, TopCache tc, const unsigned long long *__restrict__ u, int64_t k, float beta, int normalise,
     int64_t *__restrict__ idx_out, float *__restrict__ w_out, int vec_ok) {
-    __shared__ unsigned long long s_top[kTopCap];
+    __shared__ __align__(128) unsigned long long s_top[kTopCap];
+    __shared__ __align__(8) uint64_t s_bar;
     __shared__ int s_last;
     __shared__ unsigned int s_qmin; // smallest mass drawn by this block
     const int lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) s_qmin = 0xffffffffu;
+    // One thread pulls the cached levels in with bulk asynchronous copies (one round trip for all of
+    // them); sizes are rounded up to 16 bytes, the slack lies inside the levels' 256-byte padding.
+    if (threadIdx.x == 0) {
+        s_qmin = 0xffffffffu;
+        mbar_init(&s_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        unsigned int bytes = 0;
+        for (int l = tc.from; l <= t.levels; ++l) bytes += (unsigned int)((t.count[l] + 1) & ~(int64_t)1) * 8u;
+        mbar_expect_tx(&s_bar, bytes);
+        for (int l = tc.from; l <= t.levels; ++l)
+            bulk_load(&s_top[tc.off[l]], t.lvl[l], (unsigned int)((t.count[l] + 1) & ~(int64_t)1) * 8u, &s_bar);
+    }
     const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const unsigned long long uj = (j < k) ? __ldg(u + j) : 0ull; // in flight while the cache fills
-    for (int l = tc.from; l <= t.levels; ++l) {
-#pragma unroll 4
-        for (int i = threadIdx.x; i < t.count[l]; i += blockDim.x) s_top[tc.off[l] + i] = __ldcg(&t.lvl[l][i]);
+    __syncthreads(); // the barrier object is initialised
+    {
+        unsigned int spins = 0;
+        while (!mbar_try_wait(&s_bar, 0u)) {
+            if (++spins > (1u << 24)) { // a copy never landed: report, carry on with what is there
+                if (threadIdx.x == 0) set_status(&t.hdr->status, DISTRL_ERR_TIMEOUT);
+                break;
+            }
+        }
     }
-    __syncthreads();
     if (j < k) {
         // top level: its entries sum to the total mass
         int l = t.levels;
@@ -239,13 +275,14 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     __syncthreads();
     if (threadIdx.x == 0) {
         atomicMin(&t.hdr->qmin, s_qmin);
-        __threadfence();
-        unsigned int done = atomicAdd(&t.hdr->done, 1u);
+        // release: this block's parked masses and its minimum are visible to whoever sees the count;
+        // acquire: the last block sees everybody else's
+        unsigned int done;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(done) : "l"(&t.hdr->done) : "memory");
         s_last = (done == gridDim.x - 1);
     }
     __syncthreads();
     if (!s_last) return;
-    __threadfence();
     const double qmin = (double)atomicMin(&t.hdr->qmin, 0xffffffffu); // atomic read
     for (int64_t i0 = threadIdx.x; i0 < k; i0 += 4 * (int64_t)blockDim.x) { // four loads in flight per thread
         uint32_t qs[4];
@@ -339,8 +376,12 @@ __global__ void __launch_bounds__(kUpdateThreads) update_apply_kernel(Tree t, Up
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j < k) {
         const int64_t i = idx[j];
-        if (i >= 0 && i < t.n && __ldcg(uw.claim + i) == (unsigned int)j) {
-            const uint32_t qn = uw.newq[j], qo = __ldcg(t.q + i);
+        const bool in = (i >= 0 && i < t.n);
+        // claim and old mass are fetched together; the old mass is only used by the winner
+        const unsigned int cl = in ? __ldcg(uw.claim + i) : 0xffffffffu;
+        const uint32_t qo = in ? __ldcg(t.q + i) : 0u;
+        if (in && cl == (unsigned int)j) {
+            const uint32_t qn = uw.newq[j];
             if (qn != qo) {
                 t.q[i] = qn;
                 const unsigned long long diff = (unsigned long long)qn - (unsigned long long)qo; // mod 2^64
@@ -398,9 +439,10 @@ extern "C" int distrl_build_sampler(uint32_t *prio_q, int64_t n, void *workspace
         tc.from = s->tree.levels + 1;
         tc.total = 0;
         for (int l = s->tree.levels; l >= 1; --l) {
-            if (tc.total + s->tree.count[l] > kTopCap) break;
+            const int padded = (int)((s->tree.count[l] + 1) & ~(int64_t)1); // whole 16-byte units
+            if (tc.total + padded > kTopCap) break;
             tc.off[l] = tc.total;
-            tc.total += (int)s->tree.count[l];
+            tc.total += padded;
             tc.from = l;
         }
     }

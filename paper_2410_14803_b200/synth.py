@@ -88,10 +88,12 @@ def _lengths_to_total(rng, n, draw):
     return lens
 
 
-def make_workload(index: int, n_override: Optional[int] = None, m_override: Optional[int] = None) -> Workload:
-    """Build workload `index` (0..4); the overrides shrink it for tests while keeping its recipe."""
+def make_workload(index: int, n_override: Optional[int] = None, m_override: Optional[int] = None,
+                  shard: int = 0) -> Workload:
+    """Build workload `index` (0..4); the overrides shrink it for tests while keeping its recipe.
+    `shard` > 0 gives an independent buffer of the same recipe (one per GPU in multi-GPU runs)."""
     spec = dict(_SPECS[index])
-    rng = np.random.Generator(np.random.PCG64(BASE_SEED + index))
+    rng = np.random.Generator(np.random.PCG64(BASE_SEED + index + 100000 * shard))
     n_fixed = n_override if (n_override is not None and spec["n"] is not None) else spec["n"]
     tmax = spec["tmax"]
     if index == 3:
