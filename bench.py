@@ -196,15 +196,16 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     w = synth.make_workload(WORKLOAD_INDEX[args.workload], shard=rank)   # every rank owns its own shard
-    if w.token_level:
-        raise SystemExit("token-level workload: use tests; bench times the fp32 workloads")
     a = w.arrays
     n, k, R = w.n, w.batch, w.rounds
     cfg = distrl.make_prio_cfg(w.w_td, w.w_rho, w.w_ent, w.rho_clip, w.alpha, w.scale)
 
     # ---- host (pinned) copies: the e2e leg starts from these every step
-    names = ["traj_offsets", "rewards", "values", "logp_target", "logp_behaviour", "entropy"]
-    host = {nm: torch.from_numpy(a[nm]).pin_memory() for nm in names}
+    tok = w.token_level
+    names = ["traj_offsets", "rewards", "values", "entropy"] + \
+            (["step_token_offsets", "tok_logp_target", "tok_logp_behaviour"] if tok else ["logp_target", "logp_behaviour"])
+    as_t = lambda nm: torch.from_numpy(a[nm]).view(torch.bfloat16) if nm.startswith("tok_") else torch.from_numpy(a[nm])
+    host = {nm: as_t(nm).pin_memory() for nm in names}
     u_all = np.stack([synth.uniforms(w, r) for r in range(R)]).view(np.int64)
     nd_all = np.stack([synth.fresh_abs_delta(w, r) for r in range(R)])
     host_u, host_nd = torch.from_numpy(u_all).pin_memory(), torch.from_numpy(nd_all).pin_memory()
@@ -221,12 +222,19 @@ def run_ours(args):
     ws_s = distrl.alloc_workspace(distrl.distrl_sampler_workspace_bytes(n))
     distrl.distrl_workspace_init(ws_r)
     distrl.distrl_workspace_init(ws_s)
-    batch = distrl.make_batch(dv["traj_offsets"], dv["rewards"], dv["values"], dv["logp_target"], dv["logp_behaviour"])
+    if tok:   # per-step log-probs are the token sums the Retrace pass writes out
+        lp_buf, lm_buf = f32(), f32()
+        batch = distrl.make_batch(dv["traj_offsets"], dv["rewards"], dv["values"], None, None, None,
+                                  dv["step_token_offsets"], dv["tok_logp_target"], dv["tok_logp_behaviour"])
+    else:
+        lp_buf, lm_buf = dv["logp_target"], dv["logp_behaviour"]
+        batch = distrl.make_batch(dv["traj_offsets"], dv["rewards"], dv["values"], lp_buf, lm_buf)
+    lp_out, lm_out = (lp_buf, lm_buf) if tok else (None, None)
 
     # The heavy-tailed critic error of workload 3 is workload synthesis, not part of the method: the
     # scaled |delta| array that the priority stage reads is prepared once from the same td_delta the
     # Retrace stage writes every step (bit-identical each step), so no foreign kernel runs in the timed region.
-    distrl.distrl_retrace_targets(batch, w.gamma, w.lam, vt, adv, dl, workspace=ws_r)
+    distrl.distrl_retrace_targets(batch, w.gamma, w.lam, vt, adv, dl, lp_out, lm_out, workspace=ws_r)
     prio_in = (dl * tail) if tail is not None else dl
     torch.cuda.synchronize()
 
@@ -236,8 +244,7 @@ def run_ours(args):
     def rounds(s):
         for r in range(R):
             distrl.distrl_sample(s, d_u[r], w.beta, True, idx[r], wts[r])
-            distrl.distrl_update_priorities(s, idx[r], d_nd[r], dv["logp_target"], dv["logp_behaviour"],
-                                            dv["entropy"], cfg, None)
+            distrl.distrl_update_priorities(s, idx[r], d_nd[r], lp_buf, lm_buf, dv["entropy"], cfg, None)
 
     # The R sample->refresh rounds are launch-bound (3 short kernels each), so the caller records them once
     # into a CUDA graph and replays it every step.  The sampler handle only holds pointers into ws_s and q,
@@ -255,9 +262,9 @@ def run_ours(args):
 
     def step(marks=None):
         if marks: marks[0].record()
-        distrl.distrl_retrace_targets(batch, w.gamma, w.lam, vt, adv, dl, workspace=ws_r)
+        distrl.distrl_retrace_targets(batch, w.gamma, w.lam, vt, adv, dl, lp_out, lm_out, workspace=ws_r)
         if marks: marks[1].record()
-        distrl.distrl_compute_priorities(prio_in, dv["logp_target"], dv["logp_behaviour"], dv["entropy"], cfg, None, q)
+        distrl.distrl_compute_priorities(prio_in, lp_buf, lm_buf, dv["entropy"], cfg, None, q)
         if marks: marks[2].record()
         s = distrl.distrl_build_sampler(q, ws_s)
         if marks: marks[3].record()
@@ -336,7 +343,10 @@ def run_ours(args):
         return 0
 
     peak, peak_kind = _peaks()
-    retrace_bytes = 28 * n + 8 * (w.m + 1)       # r, V, logpi, logmu in; v_target, advantage, td_delta out; offsets
+    if tok:   # r, V, step offsets, both bf16 token arrays in; v_target, advantage, td_delta, logpi, logmu out; offsets
+        retrace_bytes = (8 + 8 + 20) * n + 4 * int(a["step_token_offsets"][-1]) + 8 * (w.m + 1)
+    else:     # r, V, logpi, logmu in; v_target, advantage, td_delta out; offsets
+        retrace_bytes = 28 * n + 8 * (w.m + 1)
     prio_bytes = 20 * n                          # delta, logpi, logmu, entropy in; q out
     build_bytes = 4 * n + 8 * (n // 128)
     ach = retrace_bytes / (stage_ms[0] * 1e-3) / 1e9
@@ -354,7 +364,7 @@ def run_ours(args):
             "priorities_gbs": prio_bytes / (stage_ms[1] * 1e-3) / 1e9,
             "build_sampler_gbs": build_bytes / (stage_ms[2] * 1e-3) / 1e9,
         },
-        "roofline": {"bound": "hbm", "kernel": "scan_kernel (distrl_retrace_targets)", "achieved": ach, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "scan_prep_kernel + %s (distrl_retrace_targets)" % ("scan_kernel<4,tokens>" if tok else "scan_pipe_kernel"), "achieved": ach, "peak": peak,
                      "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
                      "frac_of_nominal_8000": ach / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH,
                      "algorithmic_bytes": retrace_bytes},

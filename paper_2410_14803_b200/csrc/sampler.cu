@@ -261,7 +261,6 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
             idx_out[j] = idx;
             if (w_out) {
                 if (normalise) {
-                    atomicMin(&s_qmin, qs);          // one global atomic per block, below
                     w_out[j] = __uint_as_float(qs); // parked here until the batch minimum is known
                 } else {
                     w_out[j] = powf((float)((double)t.n * (double)qs / (double)total), -beta);
@@ -270,12 +269,12 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
         }
     }
     if (!(w_out && normalise)) return;
-    // The block that finishes last divides by the batch maximum.  The largest
-    // weight belongs to the smallest sampled mass, so w_j = (q_j / q_min)^-beta.
+    // The block that finishes last divides by the batch maximum.  The largest weight belongs to the
+    // smallest sampled mass, so w_j = (q_j / q_min)^-beta; that block finds q_min among the parked
+    // masses itself, so the other blocks pay a single atomic each.
     __syncthreads();
     if (threadIdx.x == 0) {
-        atomicMin(&t.hdr->qmin, s_qmin);
-        // release: this block's parked masses and its minimum are visible to whoever sees the count;
+        // release: this block's parked masses are visible to whoever sees the count;
         // acquire: the last block sees everybody else's
         unsigned int done;
         asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(done) : "l"(&t.hdr->done) : "memory");
@@ -283,7 +282,12 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     }
     __syncthreads();
     if (!s_last) return;
-    const double qmin = (double)atomicMin(&t.hdr->qmin, 0xffffffffu); // atomic read
+    unsigned int local_min = 0xffffffffu;
+    for (int64_t i = threadIdx.x; i < k; i += blockDim.x) local_min = min(local_min, __float_as_uint(__ldcg(w_out + i)));
+    local_min = __reduce_min_sync(0xffffffffu, local_min);
+    if (lane == 0) atomicMin(&s_qmin, local_min);
+    __syncthreads();
+    const double qmin = (double)s_qmin;
     for (int64_t i0 = threadIdx.x; i0 < k; i0 += 4 * (int64_t)blockDim.x) { // four loads in flight per thread
         uint32_t qs[4];
 #pragma unroll
@@ -297,11 +301,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
             if (i < k) w_out[i] = powf((float)((double)qs[e] / qmin), -beta);
         }
     }
-    __syncthreads();
-    if (threadIdx.x == 0) { // ready for the next call
-        t.hdr->qmin = 0xffffffffu;
-        t.hdr->done = 0u;
-    }
+    if (threadIdx.x == 0) t.hdr->done = 0u; // ready for the next call
 }
 
 // ---------------------------------------------------------------------------

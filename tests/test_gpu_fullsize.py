@@ -1,0 +1,93 @@
+"""Full-size parity cases: the workloads at their real sizes, checked on sampled trajectories that the
+oracle evaluates one by one, plus properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2410_14803_b200 as distrl
+from paper_2410_14803_b200 import synth
+
+from helpers import assert_close, dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _pick_trajectories(off, n_random, tile, seed):
+    """Trajectory indices: random ones, the first and last few, and ones that straddle tile boundaries."""
+    m = off.shape[0] - 1
+    rng = np.random.default_rng(seed)
+    picks = [rng.integers(0, m, n_random), np.arange(0, 40), np.arange(m - 40, m)]
+    n = int(off[-1])
+    cuts = rng.integers(1, n // tile, 400) * tile            # transitions sitting on tile boundaries
+    picks.append(np.searchsorted(off, cuts, side="right") - 1)
+    picks.append(np.searchsorted(off, cuts - 1, side="right") - 1)
+    return np.unique(np.clip(np.concatenate(picks), 0, m - 1))
+
+
+def test_token_level_full_size_sampled_trajectories():
+    w = synth.make_workload(4)                               # 67,108,864 steps, ~1.1e9 tokens
+    a = w.arrays
+    n, off, sto = w.n, a["traj_offsets"], a["step_token_offsets"]
+    t_off, t_r, t_V, t_sto = dev(off), dev(a["rewards"]), dev(a["values"]), dev(sto)
+    t_tp = dev(a["tok_logp_target"], torch.bfloat16)
+    t_tm = dev(a["tok_logp_behaviour"], torch.bfloat16)
+    batch = distrl.make_batch(t_off, t_r, t_V, None, None, None, t_sto, t_tp, t_tm)
+    vt, adv, dl, lpo, lmo = (torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(5))
+    ws = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws)
+    distrl.distrl_retrace_targets(batch, w.gamma, w.lam, vt, adv, dl, lpo, lmo, workspace=ws)
+    assert distrl.distrl_get_status(ws) == 0
+
+    # properties that hold everywhere: at a trajectory's last step Delta = delta exactly; v_target = V + Delta
+    last = t_off[1:] - 1
+    assert torch.equal(adv[last], dl[last])
+    assert torch.all(torch.isfinite(vt)) and torch.all(torch.isfinite(adv))
+    assert float((vt - (t_V + adv)).abs().max()) <= 1e-6
+
+    # sampled trajectories, evaluated by the oracle on their own
+    js = _pick_trajectories(off, 3000, 1024, 4)
+    idx = np.concatenate([np.arange(off[j], off[j + 1]) for j in js])
+    sub_off = np.concatenate([[0], np.cumsum(off[js + 1] - off[js])]).astype(np.int64)
+    tok_idx = np.concatenate([np.arange(sto[off[j]], sto[off[j + 1]]) for j in js])
+    cnt = sto[idx + 1] - sto[idx]
+    sub_sto = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int64)
+    lp = oracle.token_logp(sub_sto, oracle.bf16_bits_to_f64(a["tok_logp_target"][tok_idx]))
+    lm = oracle.token_logp(sub_sto, oracle.bf16_bits_to_f64(a["tok_logp_behaviour"][tok_idx]))
+    o_vt, o_adv, o_dl = oracle.retrace(sub_off, a["rewards"][idx], a["values"][idx], lp, lm, w.gamma, w.lam)
+    g = torch.from_numpy(idx).cuda()
+    assert_close(lpo[g].cpu().numpy(), lp, "token logp_target")
+    assert_close(lmo[g].cpu().numpy(), lm, "token logp_behaviour")
+    assert_close(vt[g].cpu().numpy(), o_vt, "v_target")
+    assert_close(adv[g].cpu().numpy(), o_adv, "advantage")
+    assert_close(dl[g].cpu().numpy(), o_dl, "td_delta")
+
+    # the rest of the path on this buffer: priorities from the device's own sums, sampler, one round
+    cfg = distrl.make_prio_cfg(w.w_td, w.w_rho, w.w_ent, w.rho_clip, w.alpha, w.scale)
+    ent = dev(a["entropy"])
+    del t_tp, t_tm
+    mass = torch.empty(n, dtype=torch.float32, device="cuda")
+    q = torch.empty(n, dtype=torch.int32, device="cuda")
+    distrl.distrl_compute_priorities(dl, lpo, lmo, ent, cfg, mass, q)
+    o_mass = oracle.priority_mass(o_dl, lp, lm, a["entropy"][idx], w.w_td, w.w_rho, w.w_ent, w.rho_clip, w.alpha)
+    assert_close(mass[g].cpu().numpy(), o_mass, "prio_mass")
+    qh = q.cpu().numpy().view(np.uint32)
+    np.testing.assert_array_equal(qh[idx], oracle.quantise(mass[g].cpu().numpy(), w.scale))
+    ws2 = distrl.alloc_workspace(distrl.distrl_sampler_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws2)
+    s = distrl.distrl_build_sampler(q, ws2)
+    C, total = oracle.prefix(qh)
+    tot = torch.zeros(1, dtype=torch.int64, device="cuda")
+    distrl.distrl_sampler_total(s, tot)
+    assert int(tot.cpu().numpy().view(np.uint64)[0]) == total
+    u = synth.uniforms(w, 0)
+    d_idx = torch.empty(w.batch, dtype=torch.int64, device="cuda")
+    d_w = torch.empty(w.batch, dtype=torch.float32, device="cuda")
+    distrl.distrl_sample(s, dev(u.view(np.int64)), w.beta, True, d_idx, d_w)
+    y = np.array([(int(x) * total) >> 64 for x in u], dtype=np.uint64)
+    want = np.searchsorted(C, y, side="right").astype(np.int64)
+    np.testing.assert_array_equal(d_idx.cpu().numpy(), want)
+    np.testing.assert_array_equal(want[:3], oracle.sample_linear(qh, u[:3]))   # the definition itself
+    assert_close(d_w.cpu().numpy(), oracle.is_weights(qh, want, w.beta, True), "is_weight")
+    assert distrl.distrl_get_status(ws2) == 0
+    s.close()
