@@ -25,6 +25,27 @@ static inline bool aligned_to(const void *p, size_t a) {
 static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
+// Launch with programmatic stream serialisation: the grid may be scheduled while the previous kernel of
+// the stream is still draining.  Every kernel launched this way calls grid_dependency_wait() before it
+// touches global memory, so it observes exactly what an ordinary launch would.
+#ifdef __CUDACC__
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                     Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // Every workspace starts with this header (256 bytes reserved).
 struct WorkspaceHeader {
     int status;          // sticky device-side status word (distrl_status)
@@ -46,6 +67,11 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
 __device__ __forceinline__ void st_release_u32(unsigned int *p, unsigned int v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+
+// Wait until the kernels this grid depends on have completed and their writes are visible (a no-op for
+// an ordinary launch); let the kernel that follows in the stream be scheduled early.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Records the first device-side error; later ones are dropped.
 __device__ __forceinline__ void set_status(int *status, int code) { atomicCAS(status, 0, code); }

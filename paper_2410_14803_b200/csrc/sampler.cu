@@ -195,6 +195,8 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     __shared__ int s_last;
     __shared__ unsigned int s_qmin; // smallest mass drawn by this block
     const int lane = threadIdx.x & 31;
+    grid_dependency_wait();
+    grid_launch_dependents();
     // One thread pulls the cached levels in with bulk asynchronous copies (one round trip for all of
     // them); sizes are rounded up to 16 bytes, the slack lies inside the levels' 256-byte padding.
     if (threadIdx.x == 0) {
@@ -329,6 +331,8 @@ __global__ void __launch_bounds__(kUpdateThreads) update_claim_kernel(
     const float *__restrict__ lp, const float *__restrict__ lm, const float *__restrict__ ent, PrioCfg c,
     float *__restrict__ mass_out) {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    grid_dependency_wait();
+    grid_launch_dependents();
     if (j >= k) return;
     const int64_t i = idx[j];
     if (i < 0 || i >= t.n) {
@@ -358,6 +362,8 @@ __global__ void __launch_bounds__(kUpdateThreads) update_apply_kernel(Tree t, Up
     __shared__ unsigned long long s_acc[kAccCap]; // pending sums of the small top levels, per block
     __shared__ int s_acc_off[kMaxLevels + 2];
     __shared__ int s_acc_from, s_acc_used;
+    grid_dependency_wait();
+    grid_launch_dependents();
     if (threadIdx.x == 0) {
         int used = 0, from = t.levels + 1;
         for (int l = t.levels; l >= 1; --l) {
@@ -472,10 +478,10 @@ extern "C" int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k
     if (!u_fix || !idx_out) return DISTRL_ERR_NULL;
     if (!aligned_to(u_fix, 8) || !aligned_to(idx_out, 8) || !aligned_to(is_weight_out, 4)) return DISTRL_ERR_ALIGN;
     const int64_t blocks = ceil_div(k * 32, kSampleThreads);
-    sample_kernel<<<(unsigned)blocks, kSampleThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        s->tree, s->top, reinterpret_cast<const unsigned long long *>(u_fix), k, beta, normalise, idx_out, is_weight_out,
-        s->vec_ok);
-    DISTRL_CUDA_TRY(cudaGetLastError());
+    DISTRL_CUDA_TRY(launch_pdl(sample_kernel, dim3((unsigned)blocks), dim3(kSampleThreads), 0,
+                               static_cast<cudaStream_t>(stream), s->tree, s->top,
+                               reinterpret_cast<const unsigned long long *>(u_fix), k, beta, normalise, idx_out,
+                               is_weight_out, s->vec_ok));
     return DISTRL_OK;
 }
 
@@ -498,11 +504,11 @@ extern "C" int distrl_update_priorities(distrl_sampler *s, const int64_t *idx, i
     for (int64_t o = 0; o < k; o += kUpdateChunk) {
         const int kc = (int)((k - o < kUpdateChunk) ? (k - o) : kUpdateChunk);
         const unsigned grid = (unsigned)ceil_div(kc, kUpdateThreads);
-        update_claim_kernel<<<grid, kUpdateThreads, 0, st>>>(s->tree, s->upd, idx + o, kc, new_abs_delta + o, lp, lm,
-                                                            entropy, c, mass_out ? mass_out + o : nullptr);
-        DISTRL_CUDA_TRY(cudaGetLastError());
-        update_apply_kernel<<<grid, kUpdateThreads, 0, st>>>(s->tree, s->upd, idx + o, kc);
-        DISTRL_CUDA_TRY(cudaGetLastError());
+        DISTRL_CUDA_TRY(launch_pdl(update_claim_kernel, dim3(grid), dim3(kUpdateThreads), 0, st, s->tree, s->upd,
+                                   idx + o, kc, new_abs_delta + o, lp, lm, entropy, c,
+                                   mass_out ? mass_out + o : nullptr));
+        DISTRL_CUDA_TRY(launch_pdl(update_apply_kernel, dim3(grid), dim3(kUpdateThreads), 0, st, s->tree, s->upd,
+                                   idx + o, kc));
     }
     return DISTRL_OK;
 }
