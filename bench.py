@@ -195,7 +195,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    w = synth.make_workload(WORKLOAD_INDEX[args.workload], shard=rank)   # every rank owns its own shard
+    w = synth.make_workload(WORKLOAD_INDEX[args.workload], n_override=args.n_override, shard=rank)  # one shard per rank
     a = w.arrays
     n, k, R = w.n, w.batch, w.rounds
     cfg = distrl.make_prio_cfg(w.w_td, w.w_rho, w.w_ent, w.rho_clip, w.alpha, w.scale)
@@ -394,6 +394,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=sorted(WORKLOAD_INDEX), default="large")
+    ap.add_argument("--n-override", type=int, default=None,
+                    help="shrink a fixed-N workload to this many transitions (profiler captures; not a bench line)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch the sampling rounds one call at a time")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
