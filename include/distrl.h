@@ -231,6 +231,19 @@ int distrl_update_priorities(distrl_sampler *s, const int64_t *idx, int64_t k,
                              const float *logp_behaviour, const float *entropy,
                              const distrl_prio_cfg *cfg, float *mass_out, void *stream);
 
+/*
+ * Circular replay buffer (App. A, "Circular Replay Buffer": fixed capacity N, the
+ * write index advances as i <- (i+1) mod N and new experiences overwrite the
+ * oldest).  Overwrites the masses of the k slots head, head+1, ... (mod n) with
+ * new_q[0..k) and repairs every partial sum exactly, so sampling continues as if
+ * the sampler had been rebuilt.  The caller copies the transitions themselves
+ * into the same slots of its SoA arrays and advances its head to (head+k) mod n.
+ *   new_q : [k] device masses, each in [1, 2^32-1] (e.g. from distrl_compute_priorities).
+ * If k > n only the last n writes survive, as a sequential loop would leave it.
+ */
+int distrl_replay_overwrite(distrl_sampler *s, int64_t head, int64_t k, const uint32_t *new_q,
+                            void *stream);
+
 /* Writes total = sum_i q_i to *total_out_device (a device uint64). */
 int distrl_sampler_total(distrl_sampler *s, uint64_t *total_out_device, void *stream);
 

@@ -194,3 +194,12 @@ def update_from_mass(q, idx, mass_f32, scale):
     _load().oracle_update_from_mass(_n(q.shape[0]), _p(q), _n(idx.shape[0]), _p(idx), _p(m),
                                     _d(scale))
     return q
+
+
+def replay_overwrite(q, head, new_q):
+    """Circular-buffer overwrite of masses (App. A), in place on q; returns the next write index."""
+    assert q.dtype == np.uint32 and q.flags.c_contiguous
+    nq = np.ascontiguousarray(new_q, dtype=np.uint32)
+    lib = _load()
+    lib.oracle_replay_overwrite.restype = ctypes.c_int64
+    return int(lib.oracle_replay_overwrite(_n(q.shape[0]), _p(q), _n(head), _n(nq.shape[0]), _p(nq)))

@@ -286,3 +286,16 @@ int oracle_update_from_mass(int64_t n, uint32_t *q, int64_t k, const int64_t *id
         oracle_quantise(1, &mass_f32[j], scale, &q[idx[j]]);
     return 0;
 }
+
+/* Circular replay buffer of App. A ("Circular Replay Buffer"): the write index advances as
+ * i <- (i + 1) mod N and each new experience overwrites the slot it lands on.  Here only the masses
+ * are kept; returns the index the next write would use. */
+int64_t oracle_replay_overwrite(int64_t n, uint32_t *q, int64_t head, int64_t k, const uint32_t *new_q)
+{
+    int64_t i = head;
+    for (int64_t j = 0; j < k; ++j) {
+        q[i] = new_q[j];
+        i = (i + 1) % n;
+    }
+    return i;
+}

@@ -78,6 +78,7 @@ def _load():
         "distrl_build_sampler": (ci, [vp, i64, vp, sz, vp, ctypes.POINTER(vp)]),
         "distrl_sample": (ci, [vp, vp, i64, f32, ci, vp, vp, vp]),
         "distrl_update_priorities": (ci, [vp, vp, i64, vp, vp, vp, vp, ctypes.POINTER(distrl_prio_cfg), vp, vp]),
+        "distrl_replay_overwrite": (ci, [vp, i64, i64, vp, vp]),
         "distrl_sampler_total": (ci, [vp, vp, vp]),
         "distrl_sampler_level": (ci, [vp, ci, ctypes.POINTER(sz), ctypes.POINTER(i64)]),
         "distrl_destroy_sampler": (ci, [vp]),
@@ -255,6 +256,14 @@ def distrl_update_priorities(s: Sampler, idx, new_abs_delta, logp_target, logp_b
         s.handle, _ptr(idx, torch.int64), idx.numel(), _ptr(new_abs_delta, torch.float32),
         _ptr(logp_target, torch.float32), _ptr(logp_behaviour, torch.float32), _ptr(entropy, torch.float32),
         ctypes.byref(cfg), _ptr(mass_out, torch.float32), _stream(stream)), "distrl_update_priorities")
+
+
+def distrl_replay_overwrite(s: Sampler, head: int, new_q: torch.Tensor, stream=None):
+    """Overwrite the masses of slots head, head+1, ... (mod n) with new_q and repair the tree."""
+    if new_q.element_size() != 4:
+        raise ValueError("new_q must hold 32-bit masses")
+    _check(_load().distrl_replay_overwrite(s.handle, head, new_q.numel(), _ptr(new_q), _stream(stream)),
+           "distrl_replay_overwrite")
 
 
 def distrl_sampler_total(s: Sampler, total_out: torch.Tensor, stream=None):

@@ -408,6 +408,44 @@ __global__ void __launch_bounds__(kUpdateThreads) update_apply_kernel(Tree t, Up
         }
 }
 
+// ---------------------------------------------------------------------------
+// Circular overwrite (App. A, "Circular Replay Buffer": the write index advances as i <- (i+1) mod N and
+// new experiences replace the oldest).  The slots [a, b) receive the masses src[0 .. b-a); one warp per
+// touched leaf group stores them, recomputes the group's sum from the masses themselves and adds the
+// difference to every ancestor, so the tree again equals a rebuild.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) overwrite_kernel(Tree t, int64_t a, int64_t b, const uint32_t *__restrict__ src) {
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const int lane = threadIdx.x & 31;
+    const int64_t g = a / kLeaf + (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    if (g > (b - 1) / kLeaf) return; // warp-uniform
+    unsigned long long sum = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int64_t i = g * kLeaf + 4 * lane + e;
+        uint32_t v = 0u;
+        if (i < t.n) {
+            if (i >= a && i < b) { v = src[i - a]; t.q[i] = v; }
+            else v = __ldcg(t.q + i);
+        }
+        sum += v;
+    }
+    sum = warp_sum_u64(sum);
+    if (lane == 0) {
+        const unsigned long long old = t.lvl[1][g];
+        t.lvl[1][g] = sum; // this warp is the only writer of the group in this launch
+        const unsigned long long diff = sum - old; // mod 2^64
+        if (diff) {
+            int64_t node = g / kFan;
+            for (int l = 2; l <= t.levels; ++l) {
+                atomicAdd(&t.lvl[l][node], diff);
+                node /= kFan;
+            }
+        }
+    }
+}
+
 } // namespace distrl
 
 using namespace distrl;
@@ -509,6 +547,35 @@ extern "C" int distrl_update_priorities(distrl_sampler *s, const int64_t *idx, i
                                    mass_out ? mass_out + o : nullptr));
         DISTRL_CUDA_TRY(launch_pdl(update_apply_kernel, dim3(grid), dim3(kUpdateThreads), 0, st, s->tree, s->upd,
                                    idx + o, kc));
+    }
+    return DISTRL_OK;
+}
+
+extern "C" int distrl_replay_overwrite(distrl_sampler *s, int64_t head, int64_t k, const uint32_t *new_q,
+                                       void *stream) {
+    if (!s) return DISTRL_ERR_NULL;
+    const int64_t n = s->tree.n;
+    if (k < 0 || k > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
+    if (k == 0) return DISTRL_OK;
+    if (n == 0 || head < 0 || head >= n) return DISTRL_ERR_SIZE;
+    if (!new_q) return DISTRL_ERR_NULL;
+    if (!aligned_to(new_q, 4)) return DISTRL_ERR_ALIGN;
+    if (k > n) { // the buffer wraps more than once: only the last n writes survive
+        head = (head + (k - n)) % n;
+        new_q += (k - n);
+        k = n;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // at most two contiguous runs of slots; launched one after the other, so a leaf group that both
+    // touch (tiny buffers) is still written by one warp at a time
+    const int64_t first = (head + k <= n) ? k : n - head;
+    const int64_t runs[2][3] = {{head, head + first, 0}, {0, k - first, first}};
+    for (int r = 0; r < 2; ++r) {
+        const int64_t a = runs[r][0], b = runs[r][1];
+        if (b <= a) continue;
+        const int64_t groups = (b - 1) / kLeaf - a / kLeaf + 1;
+        DISTRL_CUDA_TRY(launch_pdl(overwrite_kernel, dim3((unsigned)ceil_div(groups * 32, 256)), dim3(256), 0, st,
+                                   s->tree, a, b, new_q + runs[r][2]));
     }
     return DISTRL_OK;
 }

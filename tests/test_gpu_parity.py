@@ -444,3 +444,23 @@ def test_token_level_unaligned_token_arrays():
     o_vt, o_adv, _ = oracle.retrace(a["traj_offsets"], r, V, lp, lm, w.gamma, w.lam)
     assert_close(vt.cpu().numpy(), o_vt, "v_target")
     assert_close(adv.cpu().numpy(), o_adv, "advantage")
+
+
+# ------------------------------------------------------- circular overwrite ---
+
+@pytest.mark.parametrize("n,head,k", [(100, 90, 30), (100, 0, 100), (5000, 4990, 4000), (5000, 17, 12000),
+                                      (1 << 20, (1 << 20) - 5, 4096), (300001, 123, 70000)])
+def test_replay_overwrite_equals_rebuild(n, head, k):
+    q = _masses(n, 5)
+    s, tq, ws = _build(q)
+    new_q = _masses(k, 6, heavy=False)
+    distrl.distrl_replay_overwrite(s, head, dev(new_q.view(np.int32)))
+    torch.cuda.synchronize()
+    oracle.replay_overwrite(q, head, new_q)
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), q)
+    _check_tree(s, q)
+    u = np.random.default_rng(n).integers(0, 1 << 64, size=200, dtype=np.uint64)
+    idx, _ = _sample(s, u, 0.4)
+    np.testing.assert_array_equal(idx, sample_by_prefix(q, u))
+    assert distrl.distrl_get_status(ws) == 0
+    s.close()

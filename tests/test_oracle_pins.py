@@ -359,3 +359,12 @@ def test_exact_rational_check_of_small_retrace():
     z = np.zeros(4)
     _, adv, _ = oracle.retrace(off, [float(x) for x in r], [float(x) for x in V], z, z, float(g), float(lam))
     assert [Fraction(x) for x in adv] == want
+
+
+def test_circular_overwrite_wraps_and_later_writes_win():
+    q = np.arange(1, 8, dtype=np.uint32)                      # capacity 7
+    nxt = oracle.replay_overwrite(q, 5, np.array([70, 71, 72, 73], dtype=np.uint32))
+    assert q.tolist() == [72, 73, 3, 4, 5, 70, 71] and nxt == 2
+    q = np.arange(1, 4, dtype=np.uint32)                      # more writes than slots: the last three survive
+    nxt = oracle.replay_overwrite(q, 1, np.arange(10, 18, dtype=np.uint32))
+    assert q.tolist() == [15, 16, 17] and nxt == 0            # slots visited 1,2,0,1,2,0,1,2
