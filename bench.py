@@ -366,7 +366,7 @@ def run_ours(args):
         },
         "roofline": {"bound": "hbm", "kernel": "scan_prep_kernel + %s (distrl_retrace_targets)" % ("scan_kernel<4,tokens>" if tok else "scan_pipe_kernel"), "achieved": ach, "peak": peak,
                      "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
-                     "frac_of_nominal_8000": ach / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH,
+                     "frac_of_nominal_8000": ach / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name) if args.n_override is None else None,
                      "algorithmic_bytes": retrace_bytes},
         "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": METRIC, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -382,9 +382,10 @@ def run_ours(args):
     return 0
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one scan_kernel launch, from the ncu capture summarised
-# under profiles/; None until a capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the Retrace call's kernels on workload "large"
+# (scan_pipe_kernel 270.59 + 147.47 MB, scan_prep_kernel 11.27 MB), from the ncu capture summarised in
+# profiles/scan_pipe_kernel_large.md.  Other workloads have no capture: reported as null.
+TRAFFIC_BYTES_PER_LAUNCH = {"large": 429_340_000}
 
 
 def main():
