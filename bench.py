@@ -121,7 +121,7 @@ def _config(w, args, l2):
             "gamma": w.gamma, "lambda": w.lam, "alpha": w.alpha, "beta": w.beta, "fixed_point_scale": w.scale,
             "parallelism": "independent replay shard per GPU (no data-path collective)" if args.gpus > 1 else "1 GPU",
             "l2": l2,
-            "rounds_launch": "eager" if getattr(args, "no_graph", False) else "caller-side CUDA graph of the rounds"}
+            "fused_pass": bool(getattr(args, "fused", False)), "rounds_launch": "eager" if getattr(args, "no_graph", False) else "caller-side CUDA graph of the rounds"}
 
 
 # --------------------------------------------------------------------------- CUDA legs
@@ -240,6 +240,8 @@ def run_ours(args):
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
     launches_per_step = 2 + 1 + 2 + 3 * R   # scan prep + scan, priorities, 2 build, (sample, claim, apply) x R
+    if args.fused:
+        launches_per_step = 3 + 3 * R       # scan prep + fused scan + upper tree levels, then the rounds
 
     def rounds(s):
         for r in range(R):
@@ -261,6 +263,19 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def step(marks=None):
+        if args.fused:   # Retrace + priorities + sampler build in one pass over the buffer
+            if marks: marks[0].record()
+            s = distrl.distrl_retrace_priorities_build(batch, w.gamma, w.lam, dv["entropy"], tail, cfg, vt, adv, None,
+                                                       q, None, retrace_workspace=ws_r, sampler_workspace=ws_s)
+            if marks:
+                marks[1].record(); marks[2].record(); marks[3].record()
+            if graph is not None:
+                graph.replay()
+            else:
+                rounds(s)
+            if marks: marks[4].record()
+            s.close()
+            return
         if marks: marks[0].record()
         distrl.distrl_retrace_targets(batch, w.gamma, w.lam, vt, adv, dl, lp_out, lm_out, workspace=ws_r)
         if marks: marks[1].record()
@@ -349,6 +364,8 @@ def run_ours(args):
         retrace_bytes = 28 * n + 8 * (w.m + 1)
     prio_bytes = 20 * n                          # delta, logpi, logmu, entropy in; q out
     build_bytes = 4 * n + 8 * (n // 128)
+    if args.fused:   # r, V, logpi, logmu, entropy (+ scale) in; v_target, advantage, q out; offsets; tree levels 1-2
+        retrace_bytes = (20 + (4 if tail is not None else 0) + 12) * n + 8 * (w.m + 1) + 8 * (n // 128)
     ach = retrace_bytes / (stage_ms[0] * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": world * n / (ms_per_step * 1e-3), "unit": METRIC, "n_gpus": world,
@@ -366,7 +383,7 @@ def run_ours(args):
         },
         "roofline": {"bound": "hbm", "kernel": "scan_prep_kernel + %s (distrl_retrace_targets)" % ("scan_kernel<4,tokens>" if tok else "scan_pipe_kernel"), "achieved": ach, "peak": peak,
                      "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
-                     "frac_of_nominal_8000": ach / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name) if args.n_override is None else None,
+                     "frac_of_nominal_8000": ach / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name) if (args.n_override is None and not args.fused) else None,
                      "algorithmic_bytes": retrace_bytes},
         "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": METRIC, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -398,6 +415,8 @@ def main():
     ap.add_argument("--n-override", type=int, default=None,
                     help="shrink a fixed-N workload to this many transitions (profiler captures; not a bench line)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fused", action="store_true",
+                    help="use distrl_retrace_priorities_build (one pass) instead of the three separate calls")
     ap.add_argument("--no-graph", action="store_true", help="launch the sampling rounds one call at a time")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()

@@ -244,6 +244,27 @@ int distrl_update_priorities(distrl_sampler *s, const int64_t *idx, int64_t k,
 int distrl_replay_overwrite(distrl_sampler *s, int64_t head, int64_t k, const uint32_t *new_q,
                             void *stream);
 
+/*
+ * Retrace targets (Section 5.2), priorities (Section 5.3) and the sampler's sum
+ * tree in ONE pass over the trajectory buffer: what distrl_retrace_targets,
+ * distrl_compute_priorities and distrl_build_sampler compute, without writing
+ * td_delta and reading it (and both log-prob arrays, and prio_q) back.
+ *   entropy     : [N] or NULL (NULL => H_t = -logpi_t).
+ *   delta_scale : [N] or NULL; the priority uses |delta_t * delta_scale[t]|.
+ *   td_delta    : [N] output or NULL;  prio_mass : [N] output or NULL.
+ *   prio_q      : [N] output, kept by the sampler like in distrl_build_sampler.
+ * Served only for fp32 per-step log-probs without bootstrap values and with
+ * every array 16-byte aligned (DISTRL_ERR_PARAM / DISTRL_ERR_ALIGN otherwise:
+ * use the three separate calls).  Results obey the same contracts as theirs.
+ */
+int distrl_retrace_priorities_build(const distrl_batch *batch, float gamma, float lambda,
+                                    const float *entropy, const float *delta_scale,
+                                    const distrl_prio_cfg *cfg, float *v_target, float *advantage,
+                                    float *td_delta, uint32_t *prio_q, float *prio_mass,
+                                    void *retrace_workspace, size_t retrace_workspace_bytes,
+                                    void *sampler_workspace, size_t sampler_workspace_bytes,
+                                    void *stream, distrl_sampler **out);
+
 /* Writes total = sum_i q_i to *total_out_device (a device uint64). */
 int distrl_sampler_total(distrl_sampler *s, uint64_t *total_out_device, void *stream);
 

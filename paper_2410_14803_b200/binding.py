@@ -78,6 +78,9 @@ def _load():
         "distrl_build_sampler": (ci, [vp, i64, vp, sz, vp, ctypes.POINTER(vp)]),
         "distrl_sample": (ci, [vp, vp, i64, f32, ci, vp, vp, vp]),
         "distrl_update_priorities": (ci, [vp, vp, i64, vp, vp, vp, vp, ctypes.POINTER(distrl_prio_cfg), vp, vp]),
+        "distrl_retrace_priorities_build": (ci, [ctypes.POINTER(distrl_batch), f32, f32, vp, vp,
+                                                 ctypes.POINTER(distrl_prio_cfg), vp, vp, vp, vp, vp, vp, sz, vp, sz, vp,
+                                                 ctypes.POINTER(vp)]),
         "distrl_replay_overwrite": (ci, [vp, i64, i64, vp, vp]),
         "distrl_sampler_total": (ci, [vp, vp, vp]),
         "distrl_sampler_level": (ci, [vp, ci, ctypes.POINTER(sz), ctypes.POINTER(i64)]),
@@ -256,6 +259,21 @@ def distrl_update_priorities(s: Sampler, idx, new_abs_delta, logp_target, logp_b
         s.handle, _ptr(idx, torch.int64), idx.numel(), _ptr(new_abs_delta, torch.float32),
         _ptr(logp_target, torch.float32), _ptr(logp_behaviour, torch.float32), _ptr(entropy, torch.float32),
         ctypes.byref(cfg), _ptr(mass_out, torch.float32), _stream(stream)), "distrl_update_priorities")
+
+
+def distrl_retrace_priorities_build(batch: distrl_batch, gamma: float, lam: float, entropy, delta_scale,
+                                    cfg: distrl_prio_cfg, v_target, advantage, td_delta, prio_q, prio_mass, *,
+                                    retrace_workspace, sampler_workspace, stream=None) -> Sampler:
+    """Retrace targets, priorities and the sampler's tree in one pass; returns the sampler."""
+    out = ctypes.c_void_p()
+    _check(_load().distrl_retrace_priorities_build(
+        ctypes.byref(batch), gamma, lam, _ptr(entropy, torch.float32), _ptr(delta_scale, torch.float32),
+        ctypes.byref(cfg), _ptr(v_target, torch.float32), _ptr(advantage, torch.float32),
+        _ptr(td_delta, torch.float32), _ptr(prio_q), _ptr(prio_mass, torch.float32), _ptr(retrace_workspace),
+        retrace_workspace.numel() * retrace_workspace.element_size(), _ptr(sampler_workspace),
+        sampler_workspace.numel() * sampler_workspace.element_size(), _stream(stream), ctypes.byref(out)),
+        "distrl_retrace_priorities_build")
+    return Sampler(out.value, prio_q, sampler_workspace)
 
 
 def distrl_replay_overwrite(s: Sampler, head: int, new_q: torch.Tensor, stream=None):

@@ -15,6 +15,7 @@
 //            winners store the new mass and add new - old to every ancestor, so
 //            the tree stays bit-identical to a rebuild.
 #include "priority.cuh"
+#include "sampler.cuh"
 
 #include <new>
 
@@ -463,8 +464,9 @@ extern "C" size_t distrl_sampler_workspace_bytes(int64_t n) {
     return tree_layout(n, nullptr, nullptr, nullptr);
 }
 
-extern "C" int distrl_build_sampler(uint32_t *prio_q, int64_t n, void *workspace, size_t workspace_bytes,
-                                    void *stream, distrl_sampler **out) {
+namespace distrl {
+
+int sampler_create(uint32_t *prio_q, int64_t n, void *workspace, size_t workspace_bytes, distrl_sampler **out) {
     if (!out) return DISTRL_ERR_NULL;
     *out = nullptr;
     if (n < 0 || n > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
@@ -493,17 +495,41 @@ extern "C" int distrl_build_sampler(uint32_t *prio_q, int64_t n, void *workspace
     s->tree.q = prio_q;
     s->vec_ok = aligned_to(prio_q, 16) ? 1 : 0;
     *out = s;
+    return DISTRL_OK;
+}
+
+void sampler_tree_base(const distrl_sampler *s, TreeBase *out) {
+    const Tree &t = s->tree;
+    out->lvl1 = t.lvl[1];
+    out->n1 = t.count[1];
+    out->lvl2 = t.levels >= 2 ? t.lvl[2] : nullptr;
+    out->n2 = t.levels >= 2 ? t.count[2] : 0;
+    out->levels = t.levels;
+    out->hdr = t.hdr;
+}
+
+int sampler_build_upper(const distrl_sampler *s, cudaStream_t st) {
+    if (s->tree.levels >= 3) {
+        build_upper_kernel<<<1, 1024, 0, st>>>(s->tree);
+        DISTRL_CUDA_TRY(cudaGetLastError());
+    }
+    return DISTRL_OK;
+}
+
+} // namespace distrl
+
+extern "C" int distrl_build_sampler(uint32_t *prio_q, int64_t n, void *workspace, size_t workspace_bytes,
+                                    void *stream, distrl_sampler **out) {
+    int rc = sampler_create(prio_q, n, workspace, workspace_bytes, out);
+    if (rc) return rc;
     if (n == 0) return DISTRL_OK;
+    distrl_sampler *s = *out;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Tree &t = s->tree;
     unsigned grid = (unsigned)(t.levels >= 2 ? t.count[2] : 1);
     build_leaf_kernel<<<grid, 256, 0, st>>>(t, s->vec_ok);
     DISTRL_CUDA_TRY(cudaGetLastError());
-    if (t.levels >= 3) {
-        build_upper_kernel<<<1, 1024, 0, st>>>(t);
-        DISTRL_CUDA_TRY(cudaGetLastError());
-    }
-    return DISTRL_OK;
+    return sampler_build_upper(s, st);
 }
 
 extern "C" int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k, float beta, int normalise,

@@ -464,3 +464,70 @@ def test_replay_overwrite_equals_rebuild(n, head, k):
     np.testing.assert_array_equal(idx, sample_by_prefix(q, u))
     assert distrl.distrl_get_status(ws) == 0
     s.close()
+
+
+# ---------------------------------------------------------------- fused pass ---
+
+@pytest.mark.parametrize("index,with_ent,with_scale,n_over", [(0, True, False, None), (1, True, True, None),
+                                                              (1, False, False, None), (2, True, True, None),
+                                                              (3, True, True, 3000001)])
+def test_fused_retrace_priorities_build(index, with_ent, with_scale, n_over):
+    w = synth.make_workload(index, n_override=n_over)
+    a = w.arrays
+    n = w.n
+    cfg = prio_cfg_of(w)
+    scale = synth.heavy_tail_scale(w) if with_scale else None
+    t = [dev(a["traj_offsets"]), dev(a["rewards"]), dev(a["values"]), dev(a["logp_target"]), dev(a["logp_behaviour"])]
+    batch = distrl.make_batch(*t)
+    t_ent = dev(a["entropy"]) if with_ent else None
+    t_sc = dev(scale) if with_scale else None
+    vt, adv, dl, mass = (torch.full((n,), float("nan"), dtype=torch.float32, device="cuda") for _ in range(4))
+    tq = torch.zeros(n, dtype=torch.int32, device="cuda")
+    ws_r = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    ws_s = distrl.alloc_workspace(distrl.distrl_sampler_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws_r)
+    distrl.distrl_workspace_init(ws_s)
+    s = distrl.distrl_retrace_priorities_build(batch, w.gamma, w.lam, t_ent, t_sc, cfg, vt, adv, dl, tq, mass,
+                                               retrace_workspace=ws_r, sampler_workspace=ws_s)
+    assert distrl.distrl_get_status(ws_r) == 0
+    o_vt, o_adv, o_dl = oracle.retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"],
+                                       a["logp_behaviour"], w.gamma, w.lam)
+    assert_close(vt.cpu().numpy(), o_vt, "v_target")
+    assert_close(adv.cpu().numpy(), o_adv, "advantage")
+    assert_close(dl.cpu().numpy(), o_dl, "td_delta")
+    d_in = o_dl * scale.astype(np.float64) if with_scale else o_dl
+    o_mass = oracle.priority_mass(d_in, a["logp_target"], a["logp_behaviour"], a["entropy"] if with_ent else None,
+                                  w.w_td, w.w_rho, w.w_ent, w.rho_clip, w.alpha)
+    assert_close(mass.cpu().numpy(), o_mass, "prio_mass")
+    q = tq.cpu().numpy().view(np.uint32)
+    np.testing.assert_array_equal(q, oracle.quantise(mass.cpu().numpy(), w.scale))
+    _check_tree(s, q)
+    u = synth.uniforms(w, 0)
+    idx, wts = _sample(s, u, w.beta)
+    np.testing.assert_array_equal(idx, sample_by_prefix(q, u))
+    assert_close(wts, oracle.is_weights(q, idx, w.beta, True), "is_weight")
+    # a refresh round on the fused sampler keeps the tree exact
+    nd = synth.fresh_abs_delta(w, 0)
+    gm = _update(s, cfg, idx, nd, t[3], t[4], t_ent if with_ent else None)
+    oracle.update_from_mass(q, idx, gm, w.scale)
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), q)
+    _check_tree(s, q)
+    assert distrl.distrl_get_status(ws_s) == 0
+    s.close()
+
+
+def test_fused_pass_refuses_what_it_does_not_serve():
+    w = synth.make_workload(0)
+    a = w.arrays
+    n = w.n
+    t = [dev(a["traj_offsets"]), dev(a["rewards"]), dev(a["values"]), dev(a["logp_target"]), dev(a["logp_behaviour"])]
+    boot = torch.zeros(w.m, dtype=torch.float32, device="cuda")
+    batch = distrl.make_batch(*t, boot)
+    out = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(2)]
+    tq = torch.zeros(n, dtype=torch.int32, device="cuda")
+    ws_r = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    ws_s = distrl.alloc_workspace(distrl.distrl_sampler_workspace_bytes(n))
+    with pytest.raises(distrl.DistrlError) as e:
+        distrl.distrl_retrace_priorities_build(batch, 0.9, 0.9, None, None, prio_cfg_of(w), out[0], out[1], None, tq,
+                                               None, retrace_workspace=ws_r, sampler_workspace=ws_s)
+    assert e.value.code == distrl.binding.ERR_PARAM
