@@ -22,20 +22,20 @@ __global__ void __launch_bounds__(kPrioThreads) priority_kernel(
             float4 ms = make_float4(prio_mass(d.x, p.x, m.x, h.x, c), prio_mass(d.y, p.y, m.y, h.y, c),
                                     prio_mass(d.z, p.z, m.z, h.z, c), prio_mass(d.w, p.w, m.w, h.w, c));
             if (mass_out) stg_stream_f4(mass_out + 4 * v, ms);
-            uint4 q = make_uint4(prio_quantise(ms.x, c.scale), prio_quantise(ms.y, c.scale),
-                                 prio_quantise(ms.z, c.scale), prio_quantise(ms.w, c.scale));
+            uint4 q = make_uint4(prio_quantise(ms.x, c), prio_quantise(ms.y, c),
+                                 prio_quantise(ms.z, c), prio_quantise(ms.w, c));
             *reinterpret_cast<uint4 *>(q_out + 4 * v) = q; // kept in L2: the sampler build reads it next
         }
         for (int64_t t = 4 * n4 + g; t < n; t += stride) {
             float ms = prio_mass(delta[t], lp[t], lm[t], ent ? ent[t] : -lp[t], c);
             if (mass_out) mass_out[t] = ms;
-            q_out[t] = prio_quantise(ms, c.scale);
+            q_out[t] = prio_quantise(ms, c);
         }
     } else {
         for (int64_t t = g; t < n; t += stride) {
             float ms = prio_mass(delta[t], lp[t], lm[t], ent ? ent[t] : -lp[t], c);
             if (mass_out) mass_out[t] = ms;
-            q_out[t] = prio_quantise(ms, c.scale);
+            q_out[t] = prio_quantise(ms, c);
         }
     }
 }
@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(kPrioThreads) priority_traj_kernel(
                 ms = (c.alpha == 0.5f) ? sqrtf(p) : (c.alpha == 1.0f) ? p : powf(p, c.alpha);
             }
             if (mass_out) mass_out[j] = ms;
-            q_out[j] = prio_quantise(ms, c.scale);
+            q_out[j] = prio_quantise(ms, c);
         }
     }
 }

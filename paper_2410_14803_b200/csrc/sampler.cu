@@ -355,7 +355,7 @@ __global__ void __launch_bounds__(kUpdateThreads) update_claim_kernel(
     }
     const float mass = prio_mass(new_abs_delta[j], p, m, h, c);
     if (mass_out) mass_out[j] = mass;
-    uw.newq[j] = prio_quantise(mass, c.scale);
+    uw.newq[j] = prio_quantise(mass, c);
 }
 
 __global__ void __launch_bounds__(kUpdateThreads) update_apply_kernel(Tree t, UpdateWs uw,
