@@ -1,0 +1,74 @@
+"""The pins are only worth something if a plausible mistake in the oracle trips one of them.
+Here mistakes are planted in copies of the oracle's C source (on the CPU, never in the CUDA path):
+each mutated copy is compiled, swapped in for the real library, and at least one pin must fail."""
+import ctypes
+import os
+import subprocess
+import tempfile
+
+import pytest
+
+import oracle
+import test_oracle_pins as pins
+
+SRC = os.path.join(os.path.dirname(os.path.abspath(oracle.__file__)), "distrl_oracle.c")
+
+PINS = [getattr(pins, n) for n in dir(pins) if n.startswith("test_")]
+
+MUTATIONS = {
+    "trace uses the step's own ratio instead of the next step's":
+        ("double Delta = last ? delta : delta + gamma * c_next * Delta_next;",
+         "double Delta = last ? delta : delta + gamma * c * Delta_next;"),
+    "ratio not truncated at one":
+        ("double c = lambda * fmin(1.0, rho);\n            double v_next", "double c = lambda * rho;\n            double v_next"),
+    "ratio inverted (mu / pi)":
+        ("double rho = exp(logp_pi[t] - logp_mu[t]);\n            double c", "double rho = exp(logp_mu[t] - logp_pi[t]);\n            double c"),
+    "discount dropped from the bootstrap term":
+        ("double delta = r[t] + gamma * v_next - V[t];", "double delta = r[t] + v_next - V[t];"),
+    "sign of V(s_t) flipped":
+        ("double delta = r[t] + gamma * v_next - V[t];", "double delta = r[t] + gamma * v_next + V[t];"),
+    "bootstrap ignored":
+        ("double v_next = last ? (boot ? boot[j] : 0.0) : V[t + 1];", "double v_next = last ? 0.0 : V[t + 1];"),
+    "trajectory ends not recognised (only the buffer's last step counts as terminal)":
+        ("int last = (t == off[j + 1] - 1);\n            double rho", "int last = (t == n - 1);\n            double rho"),
+    "priority drops the entropy term":
+        ("double p = w_td * fabs(td_delta[t]) + w_rho * fmin(rho, rho_clip) + w_ent * H;",
+         "double p = w_td * fabs(td_delta[t]) + w_rho * fmin(rho, rho_clip);"),
+    "priority uses signed delta":
+        ("double p = w_td * fabs(td_delta[t]) + w_rho * fmin(rho, rho_clip) + w_ent * H;",
+         "double p = w_td * td_delta[t] + w_rho * fmin(rho, rho_clip) + w_ent * H;"),
+    "quantiser truncates instead of rounding to even":
+        ("double rn = nearbyint(x);", "double rn = floor(x);"),
+    "quantiser has no floor of one":
+        ("q = (rn < 1.0) ? 1u : (uint32_t)rn;", "q = (uint32_t)rn;"),
+    "sampler compares with >= (off by one mass unit)":
+        ("if (run > y) { pick = i; break; }", "if (run >= y) { pick = i; break; }"),
+    "importance weight exponent has the wrong sign":
+        ("w_out[j] = pow((double)n * P, -beta);", "w_out[j] = pow((double)n * P, beta);"),
+    "refresh: first duplicate wins instead of the last":
+        ("for (int64_t j = 0; j < k; ++j) {\n        int64_t i = idx[j];", "for (int64_t j = k - 1; j >= 0; --j) {\n        int64_t i = idx[j];"),
+    "Monte-Carlo return forgets the discount":
+        ("g = r[t] + gamma * g;", "g = r[t] + g;"),
+    "circular overwrite does not wrap":
+        ("i = (i + 1) % n;", "i = (i + 1 < n) ? i + 1 : i;"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_a_planted_mistake_trips_a_pin(name, monkeypatch):
+    old, new = MUTATIONS[name]
+    text = open(SRC).read()
+    assert text.count(old) == 1, "mutation site not found exactly once: " + name
+    with tempfile.TemporaryDirectory() as d:
+        src = os.path.join(d, "mutant.c")
+        lib = os.path.join(d, "mutant.so")
+        open(src, "w").write(text.replace(old, new))
+        subprocess.check_call(["gcc", "-O1", "-std=c11", "-ffp-contract=off", "-shared", "-fPIC", "-o", lib, src, "-lm"])
+        monkeypatch.setattr(oracle, "_lib", ctypes.CDLL(lib))
+        tripped = []
+        for pin in PINS:
+            try:
+                pin()
+            except AssertionError:
+                tripped.append(pin.__name__)
+        assert tripped, "no pin noticed: " + name
