@@ -387,7 +387,7 @@ def test_token_level_workload(n):
 
 @pytest.mark.parametrize("counts", ["all32", "zeros_and_ones", "one_huge", "wide"])
 def test_token_level_count_extremes(counts):
-    # all32: every tile owns more tokens than one staging pass holds; zeros_and_ones: empty steps;
+    # all32: every tile owns more tokens than one staging pass holds (18432); zeros_and_ones: empty steps;
     # one_huge: a single step with 70,000 tokens; wide: counts up to 200.
     n = 5000
     rng = np.random.default_rng(17)
@@ -415,8 +415,9 @@ def test_token_level_single_token_steps_equal_plain_logp():
     V = rng.random(n, dtype=np.float32)
     a = gpu_retrace(off, r, V, None, None, 0.99, 0.95, tokens=(sto, tok_p, tok_m))
     b = gpu_retrace(off, r, V, synth.bf16_bits_to_f32(tok_p), synth.bf16_bits_to_f32(tok_m), 0.99, 0.95)
+    # the token path takes step sums as differences of short running sums: a few ulp of the 16-token sums
     for key in ("v_target", "advantage", "td_delta"):
-        assert_close(a[key], b[key].astype(np.float64), key, tol=1e-6)
+        assert_close(a[key], b[key].astype(np.float64), key, tol=1e-5)
 
 
 def test_token_level_unaligned_token_arrays():
