@@ -532,3 +532,61 @@ def test_fused_pass_refuses_what_it_does_not_serve():
         distrl.distrl_retrace_priorities_build(batch, 0.9, 0.9, None, None, prio_cfg_of(w), out[0], out[1], None, tq,
                                                None, retrace_workspace=ws_r, sampler_workspace=ws_s)
     assert e.value.code == distrl.binding.ERR_PARAM
+
+
+def test_rounds_replayed_from_a_cuda_graph_match_the_oracle():
+    """The benchmark records the sample -> refresh rounds once into a CUDA graph and replays it; the
+    replayed launches must leave exactly the state the oracle reaches by running the rounds in order."""
+    w = synth.make_workload(2)
+    a = w.arrays
+    n, k, R = w.n, w.batch, 6
+    cfg = prio_cfg_of(w)
+    _, _, dl = oracle.retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"],
+                              w.gamma, w.lam)
+    mass0 = oracle.priority_mass(dl, a["logp_target"], a["logp_behaviour"], a["entropy"], w.w_td, w.w_rho, w.w_ent,
+                                 w.rho_clip, w.alpha)
+    q = oracle.quantise(mass0.astype(np.float32), w.scale)
+    s, tq, ws = _build(q)
+    lp, lm, ent = dev(a["logp_target"]), dev(a["logp_behaviour"]), dev(a["entropy"])
+    us = np.stack([synth.uniforms(w, r) for r in range(R)])
+    nds = np.stack([synth.fresh_abs_delta(w, r) for r in range(R)])
+    d_u, d_nd = dev(us.view(np.int64)), dev(nds)
+    idx = torch.empty((R, k), dtype=torch.int64, device="cuda")
+    wts = torch.empty((R, k), dtype=torch.float32, device="cuda")
+    mass = torch.empty((R, k), dtype=torch.float32, device="cuda")
+
+    def rounds():
+        for r in range(R):
+            distrl.distrl_sample(s, d_u[r], w.beta, True, idx[r], wts[r])
+            distrl.distrl_update_priorities(s, idx[r], d_nd[r], lp, lm, ent, cfg, mass[r])
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        rounds()                                   # first use outside capture
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    # oracle: the same six rounds, in order, from the device's own masses
+    def oracle_rounds(qq):
+        for r in range(R):
+            np.testing.assert_array_equal(idx[r].cpu().numpy(), sample_by_prefix(qq, us[r]))
+            assert_close(wts[r].cpu().numpy(), oracle.is_weights(qq, idx[r].cpu().numpy(), w.beta, True), "is_weight")
+            oracle.update_from_mass(qq, idx[r].cpu().numpy(), mass[r].cpu().numpy(), w.scale)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        rounds()
+    torch.cuda.synchronize()
+    # state now: rounds ran once (eagerly; capture itself launches nothing)
+    q1 = q.copy()
+    # replay twice; after each replay the recorded outputs describe that replay
+    for _ in range(2):
+        q_before = tq.cpu().numpy().view(np.uint32).copy()
+        graph.replay()
+        torch.cuda.synchronize()
+        qq = q_before.copy()
+        oracle_rounds(qq)
+        np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), qq)
+        _check_tree(s, qq)
+    assert distrl.distrl_get_status(ws) == 0
+    del q1
+    s.close()
