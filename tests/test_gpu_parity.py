@@ -403,6 +403,58 @@ def test_token_level_count_extremes(counts):
     _token_case(off, sto, tok_p, tok_m, 3)
 
 
+@pytest.mark.parametrize("n", [1, 2, 511, 512, 513, 544, 545, 546, 1023, 1024, 1025, 1057, 1569, 4097])
+@pytest.mark.parametrize("kind", ["single", "ones", "tile_straddle", "long_mixed"])
+def test_token_level_tile_edges(n, kind):
+    # sizes around the 512-step tiles and the 32-step halo of the pipelined token kernel: which tiles are
+    # staged, which are taken straight from global memory, where the buffer ends inside a halo
+    rng = np.random.default_rng(1000 + n)
+    cnt = rng.integers(1, 33, n)
+    sto = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int64)
+    nt = int(sto[-1])
+    tok_m = synth.f32_to_bf16_bits((rng.standard_normal(nt) * 0.3 - 0.3).astype(np.float32))
+    tok_p = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(tok_m) + (rng.standard_normal(nt) * 0.05).astype(np.float32))
+    off = synth.adversarial_offsets(kind, n, tile=512)
+    _token_case(off, sto, tok_p, tok_m, n)
+
+
+@pytest.mark.parametrize("counts", ["first_vector_only", "sparse", "near_capacity", "over_capacity_some"])
+def test_token_level_staging_corners(counts):
+    # first_vector_only: all tokens of a tile inside one 16-byte vector; sparse: most steps empty;
+    # near_capacity: tiles just below what a stage holds; over_capacity_some: staged and direct tiles mixed
+    n = 6000
+    rng = np.random.default_rng(23)
+    cnt = {"first_vector_only": (np.arange(n) % 512 == 3).astype(np.int64) * 5,
+           "sparse": (rng.random(n) < 0.03).astype(np.int64) * rng.integers(1, 33, n),
+           "near_capacity": np.full(n, 18),
+           "over_capacity_some": np.where((np.arange(n) // 700) % 2 == 0, 8, 31)}[counts]
+    sto = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int64)
+    nt = int(sto[-1])
+    tok_m = synth.f32_to_bf16_bits((rng.standard_normal(nt) * 0.3 - 0.3).astype(np.float32))
+    tok_p = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(tok_m) + (rng.standard_normal(nt) * 0.05).astype(np.float32))
+    off = synth.adversarial_offsets("long_mixed", n, tile=512)
+    _token_case(off, sto, tok_p, tok_m, 5)
+
+
+def test_token_level_bad_step_offsets_are_reported_not_fatal():
+    n = 3000
+    rng = np.random.default_rng(3)
+    cnt = rng.integers(1, 33, n)
+    sto = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int64)
+    nt = int(sto[-1])
+    tok = synth.f32_to_bf16_bits((rng.standard_normal(nt) * 0.3 - 0.3).astype(np.float32))
+    bad = sto.copy()
+    bad[700] = bad[699] - 40          # a decreasing pair inside a staged tile
+    bad[2900] = bad[2899] - 3         # and one inside the last, direct tile
+    off = synth.adversarial_offsets("long_mixed", n, tile=512)
+    r = rng.normal(0, 1, n).astype(np.float32)
+    V = rng.random(n, dtype=np.float32)
+    out = gpu_retrace(off, r, V, None, None, 0.99, 0.95, tokens=(bad, tok, tok))
+    assert out["status"] == distrl.binding.ERR_OFFSETS
+    good = gpu_retrace(off, r, V, None, None, 0.99, 0.95, tokens=(sto, tok, tok))
+    assert good["status"] == 0
+
+
 def test_token_level_single_token_steps_equal_plain_logp():
     # one token per step: the token path must agree with the fp32-logp path on the same numbers
     n = 30000
