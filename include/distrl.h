@@ -119,7 +119,7 @@ int distrl_retrace_targets(const distrl_batch *batch, float gamma, float lambda,
  * whole GPU for its own pool, so that a further cudaMalloc fails or shrinks
  * that pool, or a step loop that must stay clear of cudaMalloc because it
  * stalls the whole device.  The scan's tile bookkeeping lives in a fixed
- * array inside the library image (about 0.6 MB, held by every GPU that loads
+ * array inside the library image (about 0.75 MB, held by every GPU that loads
  * the library until the process exits), which limits the size:
  *   n_transitions <= DISTRL_STATIC_MAX_N, else DISTRL_ERR_SIZE.
  * Arguments and results are those of distrl_retrace_targets, plus
