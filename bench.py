@@ -239,9 +239,9 @@ def run_ours(args):
     torch.cuda.synchronize()
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    launches_per_step = 2 + 1 + 2 + 3 * R   # scan prep + scan, priorities, 2 build, (sample, claim, apply) x R
+    launches_per_step = 2 + 1 + 2 + 3 * R   # end mask + scan, priorities, 2 build, (sample, claim, apply) x R
     if args.fused:
-        launches_per_step = 3 + 3 * R       # scan prep + fused scan + upper tree levels, then the rounds
+        launches_per_step = 3 + 3 * R       # end mask + fused scan + upper tree levels, then the rounds
 
     def rounds(s):
         for r in range(R):
@@ -381,7 +381,7 @@ def run_ours(args):
             "priorities_gbs": prio_bytes / (stage_ms[1] * 1e-3) / 1e9,
             "build_sampler_gbs": build_bytes / (stage_ms[2] * 1e-3) / 1e9,
         },
-        "roofline": {"bound": "hbm", "kernel": "scan_prep_kernel + %s (distrl_retrace_targets)" % ("scan_tok_pipe_kernel" if tok else "scan_pipe_kernel"), "achieved": ach, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "scan_mask_kernel + %s (distrl_retrace_targets)" % ("scan_tok_pipe_kernel" if tok else "scan_pipe_kernel"), "achieved": ach, "peak": peak,
                      "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
                      "frac_of_nominal_8000": ach / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name) if (args.n_override is None and not args.fused) else None,
                      "algorithmic_bytes": retrace_bytes},
@@ -399,10 +399,15 @@ def run_ours(args):
     return 0
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the Retrace call's kernels on workload "large"
-# (scan_pipe_kernel 270.59 + 147.47 MB, scan_prep_kernel 11.27 MB), from the ncu capture summarised in
-# profiles/scan_pipe_kernel_large.md.  Other workloads have no capture: reported as null.
-TRAFFIC_BYTES_PER_LAUNCH = {"large": 429_340_000}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the Retrace call's kernels, from the ncu captures
+# summarised under profiles/:
+#   "large": scan_pipe_kernel 270.59 + 153.01 MB and scan_mask_kernel 11.28 MB, captured at full size
+#            (profiles/scan_pipe_kernel_large.md);
+#   "token": scan_tok_pipe_kernel 344.47 + 65.91 MB on a 4,194,304-step case of the same workload, scaled by 16 to
+#            the full 67,108,864 steps (every array grows in proportion), plus the 34.6 MB of trajectory offsets
+#            that scan_mask_kernel reads (profiles/scan_tok_pipe_kernel_token.md).
+# Other workloads have no capture: reported as null.
+TRAFFIC_BYTES_PER_LAUNCH = {"large": 434_880_000, "token": 16 * 410_380_000 + 34_640_000}
 
 
 def main():
