@@ -410,6 +410,117 @@ __global__ void __launch_bounds__(kUpdateThreads) update_apply_kernel(Tree t, Up
 }
 
 // ---------------------------------------------------------------------------
+// update of a small batch in one launch.  For k <= kSmallBatch the election needs
+// no claim table and no second kernel: every block stages the batch's indices in
+// shared memory and a warp decides for its position j by looking at the positions
+// after it -- j applies its value iff no later position holds the same index,
+// which is what a sequential loop over the batch leaves.  The k^2 / 2 comparisons
+// (16-byte shared-memory loads, four indices each) cost less than a launch.
+// ---------------------------------------------------------------------------
+constexpr int kSmallBatch = 8192;       // positions the single-launch update serves
+constexpr int kSmallThreads = 512;
+constexpr int kSmallPerWarp = 2;        // batch positions per warp
+constexpr int kSmallPerBlock = (kSmallThreads / 32) * kSmallPerWarp;
+constexpr unsigned int kNoIndex = 0xffffffffu; // staged in place of an index outside [0, n)
+
+__global__ void __launch_bounds__(kSmallThreads) update_small_kernel(
+    Tree t, const int64_t *__restrict__ idx, int k, const float *__restrict__ new_abs_delta,
+    const float *__restrict__ lp, const float *__restrict__ lm, const float *__restrict__ ent, PrioCfg c,
+    float *__restrict__ mass_out) {
+    __shared__ __align__(16) unsigned int s_idx[kSmallBatch]; // low words of the batch's indices (n < 2^31 here)
+    __shared__ unsigned long long s_acc[kAccCap];             // pending sums of the small top levels, per block
+    __shared__ int s_acc_off[kMaxLevels + 2];
+    __shared__ int s_acc_from, s_acc_used;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    grid_dependency_wait();
+    grid_launch_dependents();
+    if (threadIdx.x == 0) {
+        int used = 0, from = t.levels + 1;
+        for (int l = t.levels; l >= 1; --l) {
+            if (used + t.count[l] > kAccCap) break;
+            s_acc_off[l] = used;
+            used += (int)t.count[l];
+            from = l;
+        }
+        s_acc_from = from;
+        s_acc_used = used;
+    }
+    // this block's positions first: their gathers are in flight while the batch is staged
+    const int j0 = blockIdx.x * kSmallPerBlock + warp * kSmallPerWarp;
+    int64_t my_i[kSmallPerWarp];
+    float g_val[kSmallPerWarp]; // lane 0: log pi, lane 1: log mu, lane 2: entropy, lane 3: old mass (bits), lane 4: |delta|
+#pragma unroll
+    for (int u = 0; u < kSmallPerWarp; ++u) {
+        const int j = j0 + u;
+        my_i[u] = (j < k) ? idx[j] : -1;
+        g_val[u] = 0.f;
+        if (my_i[u] >= 0 && my_i[u] < t.n) {
+            const int64_t i = my_i[u];
+            if (lane == 0) g_val[u] = __ldg(lp + i);
+            else if (lane == 1) g_val[u] = __ldg(lm + i);
+            else if (lane == 2) g_val[u] = ent ? __ldg(ent + i) : 0.f;
+            else if (lane == 3) g_val[u] = __uint_as_float(__ldcg(t.q + i));
+            else if (lane == 4) g_val[u] = new_abs_delta[j];
+        }
+    }
+    const int kpad = (k + 3) & ~3;
+    for (int p = threadIdx.x; p < kpad; p += kSmallThreads) {
+        const int64_t i = (p < k) ? idx[p] : -1;
+        s_idx[p] = (i >= 0 && i < t.n) ? (unsigned int)i : kNoIndex;
+    }
+    __syncthreads();
+    const int acc_from = s_acc_from, used = s_acc_used;
+    for (int i = threadIdx.x; i < used; i += kSmallThreads) s_acc[i] = 0ull;
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < kSmallPerWarp; ++u) {
+        const int j = j0 + u;
+        if (j >= k) break; // warp-uniform
+        const int64_t i = my_i[u];
+        if (i < 0 || i >= t.n) {
+            if (lane == 0) {
+                set_status(&t.hdr->status, DISTRL_ERR_INDEX);
+                if (mass_out) mass_out[j] = 0.f;
+            }
+            continue;
+        }
+        // does a later position hold the same index?
+        const unsigned int key = (unsigned int)i;
+        bool later = false;
+        for (int b = ((j + 1) & ~3) + 4 * lane; b < kpad; b += 128) {
+            const uint4 v = *reinterpret_cast<const uint4 *>(&s_idx[b]);
+            later |= (b > j && v.x == key) | (b + 1 > j && v.y == key) | (b + 2 > j && v.z == key) | (b + 3 > j && v.w == key);
+        }
+        later = __any_sync(0xffffffffu, later);
+        const float p = __shfl_sync(0xffffffffu, g_val[u], 0), m = __shfl_sync(0xffffffffu, g_val[u], 1);
+        const float h_in = __shfl_sync(0xffffffffu, g_val[u], 2);
+        const uint32_t qo = __float_as_uint(__shfl_sync(0xffffffffu, g_val[u], 3));
+        const float nd = __shfl_sync(0xffffffffu, g_val[u], 4);
+        if (lane == 0) {
+            const float mass = prio_mass(nd, p, m, ent ? h_in : -p, c);
+            if (mass_out) mass_out[j] = mass;
+            const uint32_t qn = prio_quantise(mass, c);
+            if (!later && qn != qo) {
+                t.q[i] = qn;
+                const unsigned long long diff = (unsigned long long)qn - (unsigned long long)qo; // mod 2^64
+                int64_t node = i / kLeaf;
+                for (int l = 1; l <= t.levels; ++l) {
+                    if (l >= acc_from) atomicAdd(&s_acc[s_acc_off[l] + (int)node], diff);
+                    else atomicAdd(&t.lvl[l][node], diff);
+                    node /= kFan;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    for (int l = acc_from; l <= t.levels; ++l)
+        for (int i = threadIdx.x; i < t.count[l]; i += kSmallThreads) {
+            unsigned long long d = s_acc[s_acc_off[l] + i];
+            if (d) atomicAdd(&t.lvl[l][i], d);
+        }
+}
+
+// ---------------------------------------------------------------------------
 // Circular overwrite (App. A, "Circular Replay Buffer": the write index advances as i <- (i+1) mod N and
 // new experiences replace the oldest).  The slots [a, b) receive the masses src[0 .. b-a); one warp per
 // touched leaf group stores them, recomputes the group's sum from the masses themselves and adds the
@@ -564,6 +675,11 @@ extern "C" int distrl_update_priorities(distrl_sampler *s, const int64_t *idx, i
         !aligned_to(entropy, 4) || !aligned_to(mass_out, 4))
         return DISTRL_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (k <= kSmallBatch && s->tree.n < ((int64_t)1 << 31)) { // one launch: the election happens in shared memory
+        DISTRL_CUDA_TRY(launch_pdl(update_small_kernel, dim3((unsigned)ceil_div(k, kSmallPerBlock)), dim3(kSmallThreads), 0,
+                                   st, s->tree, idx, (int)k, new_abs_delta, lp, lm, entropy, c, mass_out));
+        return DISTRL_OK;
+    }
     // chunks run one after another on the stream, so "later position wins" also holds across chunks
     for (int64_t o = 0; o < k; o += kUpdateChunk) {
         const int kc = (int)((k - o < kUpdateChunk) ? (k - o) : kUpdateChunk);
