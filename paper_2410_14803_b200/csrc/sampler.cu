@@ -285,14 +285,30 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     }
     __syncthreads();
     if (!s_last) return;
+    // Up to kTailKeep parked masses per thread stay in registers between the search for the minimum and
+    // the rescaling (a batch of 4096 draws is read once); longer batches are read again.
+    constexpr int kTailKeep = 8;
+    uint32_t kept[kTailKeep];
     unsigned int local_min = 0xffffffffu;
-    for (int64_t i = threadIdx.x; i < k; i += blockDim.x) local_min = min(local_min, __float_as_uint(__ldcg(w_out + i)));
+#pragma unroll
+    for (int e = 0; e < kTailKeep; ++e) {
+        const int64_t i = threadIdx.x + e * (int64_t)blockDim.x;
+        kept[e] = (i < k) ? __float_as_uint(__ldcg(w_out + i)) : 0xffffffffu;
+        local_min = min(local_min, kept[e]);
+    }
+    for (int64_t i = threadIdx.x + kTailKeep * (int64_t)blockDim.x; i < k; i += blockDim.x)
+        local_min = min(local_min, __float_as_uint(__ldcg(w_out + i)));
     local_min = __reduce_min_sync(0xffffffffu, local_min);
     if (lane == 0) atomicMin(&s_qmin, local_min);
     __syncthreads();
     const double qmin = (double)s_qmin;
-    for (int64_t i0 = threadIdx.x; i0 < k; i0 += 4 * (int64_t)blockDim.x) { // four loads in flight per thread
-        uint32_t qs[4];
+#pragma unroll
+    for (int e = 0; e < kTailKeep; ++e) {
+        const int64_t i = threadIdx.x + e * (int64_t)blockDim.x;
+        if (i < k) w_out[i] = powf((float)((double)kept[e] / qmin), -beta);
+    }
+    for (int64_t i0 = threadIdx.x + kTailKeep * (int64_t)blockDim.x; i0 < k; i0 += 4 * (int64_t)blockDim.x) {
+        uint32_t qs[4]; // four loads in flight per thread
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int64_t i = i0 + e * (int64_t)blockDim.x;
