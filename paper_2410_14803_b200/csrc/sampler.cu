@@ -444,23 +444,9 @@ __global__ void __launch_bounds__(kSmallThreads) update_small_kernel(
     const float *__restrict__ lp, const float *__restrict__ lm, const float *__restrict__ ent, PrioCfg c,
     float *__restrict__ mass_out) {
     __shared__ __align__(16) unsigned int s_idx[kSmallBatch]; // low words of the batch's indices (n < 2^31 here)
-    __shared__ unsigned long long s_acc[kAccCap];             // pending sums of the small top levels, per block
-    __shared__ int s_acc_off[kMaxLevels + 2];
-    __shared__ int s_acc_from, s_acc_used;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     grid_dependency_wait();
     grid_launch_dependents();
-    if (threadIdx.x == 0) {
-        int used = 0, from = t.levels + 1;
-        for (int l = t.levels; l >= 1; --l) {
-            if (used + t.count[l] > kAccCap) break;
-            s_acc_off[l] = used;
-            used += (int)t.count[l];
-            from = l;
-        }
-        s_acc_from = from;
-        s_acc_used = used;
-    }
     // this block's positions first: their gathers are in flight while the batch is staged
     const int j0 = blockIdx.x * kSmallPerBlock + warp * kSmallPerWarp;
     int64_t my_i[kSmallPerWarp];
@@ -484,9 +470,6 @@ __global__ void __launch_bounds__(kSmallThreads) update_small_kernel(
         const int64_t i = (p < k) ? idx[p] : -1;
         s_idx[p] = (i >= 0 && i < t.n) ? (unsigned int)i : kNoIndex;
     }
-    __syncthreads();
-    const int acc_from = s_acc_from, used = s_acc_used;
-    for (int i = threadIdx.x; i < used; i += kSmallThreads) s_acc[i] = 0ull;
     __syncthreads();
 #pragma unroll
     for (int u = 0; u < kSmallPerWarp; ++u) {
@@ -521,19 +504,12 @@ __global__ void __launch_bounds__(kSmallThreads) update_small_kernel(
                 const unsigned long long diff = (unsigned long long)qn - (unsigned long long)qo; // mod 2^64
                 int64_t node = i / kLeaf;
                 for (int l = 1; l <= t.levels; ++l) {
-                    if (l >= acc_from) atomicAdd(&s_acc[s_acc_off[l] + (int)node], diff);
-                    else atomicAdd(&t.lvl[l][node], diff);
+                    atomicAdd(&t.lvl[l][node], diff); // result unused: a reduction the thread does not wait for
                     node /= kFan;
                 }
             }
         }
     }
-    __syncthreads();
-    for (int l = acc_from; l <= t.levels; ++l)
-        for (int i = threadIdx.x; i < t.count[l]; i += kSmallThreads) {
-            unsigned long long d = s_acc[s_acc_off[l] + i];
-            if (d) atomicAdd(&t.lvl[l][i], d);
-        }
 }
 
 // ---------------------------------------------------------------------------
