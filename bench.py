@@ -427,7 +427,7 @@ def run_ours(args):
             "priorities_gbs": prio_bytes / (stage_ms[1] * 1e-3) / 1e9,
             "build_sampler_gbs": build_bytes / (stage_ms[2] * 1e-3) / 1e9,
         },
-        "roofline": {"bound": "hbm", "kernel": "scan_mask_kernel + %s (distrl_retrace_targets)" % ("scan_tok_pipe_kernel" if tok else "scan_pipe_kernel"), "achieved": ach, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": ("scan_mask_kernel + scan_pipe_kernel<fused> (distrl_retrace_priorities_build)" if args.fused else "scan_mask_kernel + %s (distrl_retrace_targets)" % ("scan_tok_pipe_kernel" if tok else "scan_pipe_kernel")), "achieved": ach, "peak": peak,
                      "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
                      "frac_of_nominal_8000": ach / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name) if (args.n_override is None and not args.fused) else None,
                      "algorithmic_bytes": retrace_bytes},
