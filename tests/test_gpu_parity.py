@@ -569,6 +569,41 @@ def test_fused_retrace_priorities_build(index, with_ent, with_scale, n_over):
     s.close()
 
 
+def test_fused_pass_quantiser_edges():
+    # one-step trajectories with V = 0, weights (1, 0, 0), alpha = 0.5: the priority is |r| itself, so the
+    # rewards below walk the fused epilogue through zero, a denormal, the ties of the quantiser, values
+    # that saturate it, infinity and NaN.  Whatever mass the device reports, its mass must be Q of it.
+    special = np.array([0.0, 1e-45, 1e-38, 2.0 ** -42, (1.5 * 2.0 ** -20) ** 2, (2.5 * 2.0 ** -20) ** 2, 1.0, 4096.0 ** 2,
+                        1.7e7, 3e38, np.inf, np.nan, -3.0], dtype=np.float32)
+    n = 5000
+    rng = np.random.default_rng(4)
+    r = (rng.random(n, dtype=np.float32) * 4).astype(np.float32)
+    r[:special.shape[0]] = special
+    r[2048:2048 + special.shape[0]] = special[::-1]
+    off = np.arange(n + 1, dtype=np.int64)
+    z = np.zeros(n, dtype=np.float32)
+    t = [dev(off), dev(r), dev(z), dev(z), dev(z)]
+    vt, adv, mass = (torch.full((n,), float("nan"), dtype=torch.float32, device="cuda") for _ in range(3))
+    tq = torch.zeros(n, dtype=torch.int32, device="cuda")
+    ws_r = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    ws_s = distrl.alloc_workspace(distrl.distrl_sampler_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws_r)
+    distrl.distrl_workspace_init(ws_s)
+    cfg = distrl.make_prio_cfg(1.0, 0.0, 0.0, 2.0, 0.5, 2.0 ** 20)
+    s = distrl.distrl_retrace_priorities_build(distrl.make_batch(*t), 0.9, 0.9, None, None, cfg, vt, adv, None, tq, mass,
+                                               retrace_workspace=ws_r, sampler_workspace=ws_s)
+    assert distrl.distrl_get_status(ws_r) == 0
+    q = tq.cpu().numpy().view(np.uint32)
+    m = mass.cpu().numpy()
+    np.testing.assert_array_equal(q, oracle.quantise(m, 2.0 ** 20))
+    assert q.min() >= 1
+    finite = np.isfinite(r) & (r >= 0)
+    assert_close(m[finite], np.sqrt(r[finite].astype(np.float64)), "mass of the finite rewards")
+    assert q[0] == 1 and q[6] == 1 << 20 and q[7] == 4294967295 and q[10] == 4294967295 and q[11] == 1
+    _check_tree(s, q)
+    s.close()
+
+
 def test_fused_pass_refuses_what_it_does_not_serve():
     w = synth.make_workload(0)
     a = w.arrays
