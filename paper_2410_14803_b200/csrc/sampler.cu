@@ -107,6 +107,7 @@ __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v)
 __global__ void __launch_bounds__(256) build_leaf_kernel(Tree t, int vec_ok) {
     __shared__ unsigned long long s_l1[kFan];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    grid_launch_dependents(); // pass 2 may be scheduled now; it waits for this grid before it reads
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         t.hdr->qmin = 0xffffffffu;
         t.hdr->done = 0u;
@@ -147,16 +148,17 @@ __global__ void __launch_bounds__(256) build_leaf_kernel(Tree t, int vec_ok) {
     }
 }
 
-// build, pass 2: levels 3.. from level 2, one block.
+// build, pass 2: levels 3.. from level 2, one block; one warp per entry (32 children, one coalesced
+// load).  Launched with programmatic stream serialisation: it is scheduled while pass 1 drains.
 __global__ void __launch_bounds__(1024) build_upper_kernel(Tree t) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    grid_dependency_wait();
     for (int l = 3; l <= t.levels; ++l) {
-        for (int64_t i = threadIdx.x; i < t.count[l]; i += blockDim.x) {
-            unsigned long long s = 0;
-            for (int e = 0; e < kFan; ++e) {
-                int64_t c = i * kFan + e;
-                if (c < t.count[l - 1]) s += t.lvl[l - 1][c];
-            }
-            t.lvl[l][i] = s;
+        for (int64_t e = warp; e < t.count[l]; e += 32) {
+            const int64_t ch = e * kFan + lane;
+            unsigned long long v = (ch < t.count[l - 1]) ? __ldcg(&t.lvl[l - 1][ch]) : 0ull;
+            v = warp_sum_u64(v);
+            if (lane == 0) t.lvl[l][e] = v;
         }
         __syncthreads();
     }
@@ -613,8 +615,7 @@ void sampler_tree_base(const distrl_sampler *s, TreeBase *out) {
 
 int sampler_build_upper(const distrl_sampler *s, cudaStream_t st) {
     if (s->tree.levels >= 3) {
-        build_upper_kernel<<<1, 1024, 0, st>>>(s->tree);
-        DISTRL_CUDA_TRY(cudaGetLastError());
+        DISTRL_CUDA_TRY(launch_pdl(build_upper_kernel, dim3(1), dim3(1024), 0, st, s->tree));
     }
     return DISTRL_OK;
 }
