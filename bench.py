@@ -395,6 +395,41 @@ def run_ours(args):
         barrier()
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
+    # ---- the entry points beyond the main path, each timed alone on the same buffer (not part of `value`):
+    # Monte-Carlo returns + labels, trajectory-level priorities, and a circular overwrite of 2^20 slots
+    next_rows = None
+    if args.next_rows and not tok:
+        def timed(fn, reps=20):
+            for _ in range(3):
+                fn()
+            t0, t1 = ev(), ev()
+            torch.cuda.synchronize()
+            t0.record()
+            for _ in range(reps):
+                fn()
+            t1.record()
+            torch.cuda.synchronize()
+            return t0.elapsed_time(t1) / reps * 1e-3
+        ins = main_set
+        g_ret, lab = f32(), torch.empty(n, dtype=torch.uint8, device="cuda")
+        t_mc = timed(lambda: distrl.distrl_mc_returns(ins.batch, w.gamma, g_ret, lab, workspace=ws_r))
+        q_traj = torch.empty(w.m, dtype=torch.int32, device="cuda")
+        t_tr = timed(lambda: distrl.distrl_compute_priorities_traj(ins.dv["traj_offsets"], prio_in, ins.lp_buf, ins.lm_buf,
+                                                                   ins.dv["entropy"], cfg, None, q_traj))
+        s_tmp = distrl.distrl_build_sampler(q, ws_s)
+        k_over = min(1 << 20, n)
+        new_q = torch.randint(1, 1 << 24, (k_over,), dtype=torch.int32, device="cuda")
+        t_ov = timed(lambda: distrl.distrl_replay_overwrite(s_tmp, n - k_over // 2, new_q))
+        s_tmp.close()
+        mc_bytes, tr_bytes = 9 * n + 8 * (w.m + 1), 16 * n + 8 * (w.m + 1) + 4 * w.m
+        next_rows = {
+            "mc_returns": {"ms": t_mc * 1e3, "gbs": mc_bytes / t_mc / 1e9, "frac": mc_bytes / t_mc / 1e9 / _peaks()[0]},
+            "priorities_traj": {"ms": t_tr * 1e3, "gbs": tr_bytes / t_tr / 1e9, "frac": tr_bytes / t_tr / 1e9 / _peaks()[0]},
+            "replay_overwrite": {"slots": k_over, "ms": t_ov * 1e3, "slots_per_s": k_over / t_ov},
+        }
+        if distrl.distrl_get_status(ws_r) or distrl.distrl_get_status(ws_s):
+            raise SystemExit("device status after the extra entry points")
+
     ms_per_step = total_ms / args.steps
     from paper_2410_14803_b200.shard import max_over_ranks
     ms_per_step, e2e_ms = max_over_ranks([ms_per_step, e2e_ms], device="cuda")
@@ -436,6 +471,8 @@ def run_ours(args):
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clk,
     }
+    if next_rows is not None:
+        line["next_rows"] = next_rows
     if not args.no_cpu_baseline and world == 1:
         est, desc, _ = _oracle_sample(w, 2_000_000, draws=48)
         line["cpu_baseline"] = {"value": w.n / est, "unit": METRIC, "cores": 1, "kind": "oracle", "sample": desc}
@@ -470,6 +507,8 @@ def main():
                     help="use distrl_retrace_priorities_build (one pass) instead of the three separate calls")
     ap.add_argument("--no-graph", action="store_true", help="launch the sampling rounds one call at a time")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--next-rows", action="store_true",
+                    help="also time Monte-Carlo returns, trajectory-level priorities and a circular overwrite")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -40,37 +40,58 @@ __global__ void __launch_bounds__(kPrioThreads) priority_kernel(
     }
 }
 
-// One warp per trajectory: lanes stride over its steps, shuffle-reduce the three
-// sums, lane 0 applies the formula to the means.
+// Trajectory means: a block takes kPrioThreads consecutive trajectories, whose steps are one
+// contiguous range of the buffer.  All threads stream that range with coalesced loads, a window of
+// kTrajWindow steps at a time, and leave the three per-step terms (|delta|, min(rho, clip), H) in
+// shared memory; then every thread adds up the part of its own trajectory that lies in the window.
+// The formula is applied to the means at the end.
+constexpr int kTrajWindow = 2048;
+
 __global__ void __launch_bounds__(kPrioThreads) priority_traj_kernel(
     int64_t n, int64_t m, const int64_t *__restrict__ off, const float *__restrict__ delta,
     const float *__restrict__ lp, const float *__restrict__ lm, const float *__restrict__ ent, PrioCfg c,
     float *__restrict__ mass_out, uint32_t *__restrict__ q_out) {
-    const int lane = threadIdx.x & 31;
-    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    for (int64_t j = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); j < m; j += warps) {
-        int64_t a = off[j], b = off[j + 1];
-        if (a < 0) a = 0;
-        if (b > n) b = n;
+    __shared__ float s_d[kTrajWindow], s_r[kTrajWindow], s_h[kTrajWindow];
+    const int tid = threadIdx.x;
+    auto inside = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > n ? n : x); };
+    const int64_t chunks = (m + kPrioThreads - 1) / kPrioThreads;
+    for (int64_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) { // block-uniform
+        const int64_t j0 = chunk * kPrioThreads, j = j0 + tid;
+        const int64_t j1 = (j0 + kPrioThreads < m) ? j0 + kPrioThreads : m;
+        int64_t a = 0, b = 0;
+        if (j < m) {
+            a = inside(off[j]);
+            b = inside(off[j + 1]);
+            if (b < a) b = a;
+        }
+        const int64_t A = inside(off[j0]);
+        int64_t B = inside(off[j1]);
+        if (B < A) B = A;
         float sd = 0.f, sr = 0.f, sh = 0.f;
-        for (int64_t t = a + lane; t < b; t += 32) {
-            float p = lp[t];
-            sd += fabsf(delta[t]);
-            sr += fminf(expf(p - lm[t]), c.rho_clip);
-            sh += ent ? ent[t] : -p;
+        for (int64_t p = A; p < B; p += kTrajWindow) {
+            const int cnt = (int)((B - p < kTrajWindow) ? B - p : kTrajWindow);
+            for (int i = tid; i < cnt; i += kPrioThreads) {
+                const int64_t t = p + i;
+                const float lpt = __ldcs(lp + t);
+                s_d[i] = fabsf(__ldcs(delta + t));
+                s_r[i] = fminf(expf(lpt - __ldcs(lm + t)), c.rho_clip);
+                s_h[i] = ent ? __ldcs(ent + t) : -lpt;
+            }
+            __syncthreads();
+            const int64_t lo = (a > p) ? a : p, hi = (b < p + cnt) ? b : p + cnt;
+            for (int64_t t = lo; t < hi; ++t) {
+                sd += s_d[t - p];
+                sr += s_r[t - p];
+                sh += s_h[t - p];
+            }
+            __syncthreads();
         }
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            sd += __shfl_xor_sync(0xffffffffu, sd, d);
-            sr += __shfl_xor_sync(0xffffffffu, sr, d);
-            sh += __shfl_xor_sync(0xffffffffu, sh, d);
-        }
-        if (lane == 0) {
+        if (j < m) {
             float ms = 0.f;
             if (b > a) {
-                float inv = 1.f / (float)(b - a);
-                float p = c.w_td * (sd * inv) + c.w_rho * (sr * inv) + c.w_ent * (sh * inv);
-                ms = (c.alpha == 0.5f) ? sqrtf(p) : (c.alpha == 1.0f) ? p : powf(p, c.alpha);
+                const float inv = 1.f / (float)(b - a);
+                const float pr = c.w_td * (sd * inv) + c.w_rho * (sr * inv) + c.w_ent * (sh * inv);
+                ms = (c.alpha == 0.5f) ? sqrtf(pr) : (c.alpha == 1.0f) ? pr : powf(pr, c.alpha);
             }
             if (mass_out) mass_out[j] = ms;
             q_out[j] = prio_quantise(ms, c);
@@ -130,7 +151,7 @@ extern "C" int distrl_compute_priorities_traj(int64_t n, int64_t m, const int64_
         if (p && !aligned_to(p, 4)) return DISTRL_ERR_ALIGN;
     if (!aligned_to(off, 8)) return DISTRL_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    priority_traj_kernel<<<grid_for(m * 32, kPrioThreads, 148 * 8), kPrioThreads, 0, st>>>(
+    priority_traj_kernel<<<grid_for(m, kPrioThreads, 148 * 8), kPrioThreads, 0, st>>>(
         n, m, off, td_delta, lp, lm, entropy, c, prio_mass_out, prio_q);
     DISTRL_CUDA_TRY(cudaGetLastError());
     return DISTRL_OK;
