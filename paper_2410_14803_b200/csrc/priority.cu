@@ -70,12 +70,26 @@ __global__ void __launch_bounds__(kPrioThreads) priority_traj_kernel(
         float sd = 0.f, sr = 0.f, sh = 0.f;
         for (int64_t p = A; p < B; p += kTrajWindow) {
             const int cnt = (int)((B - p < kTrajWindow) ? B - p : kTrajWindow);
-            for (int i = tid; i < cnt; i += kPrioThreads) {
-                const int64_t t = p + i;
-                const float lpt = __ldcs(lp + t);
-                s_d[i] = fabsf(__ldcs(delta + t));
-                s_r[i] = fminf(expf(lpt - __ldcs(lm + t)), c.rho_clip);
-                s_h[i] = ent ? __ldcs(ent + t) : -lpt;
+            for (int i0 = tid; i0 < cnt; i0 += 4 * kPrioThreads) { // 16 loads in flight per thread
+                float vd[4], vp[4], vm[4], ve[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + u * kPrioThreads;
+                    const int64_t t = p + (i < cnt ? i : i0);
+                    vd[u] = __ldcs(delta + t);
+                    vp[u] = __ldcs(lp + t);
+                    vm[u] = __ldcs(lm + t);
+                    ve[u] = ent ? __ldcs(ent + t) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + u * kPrioThreads;
+                    if (i < cnt) {
+                        s_d[i] = fabsf(vd[u]);
+                        s_r[i] = fminf(expf(vp[u] - vm[u]), c.rho_clip);
+                        s_h[i] = ent ? ve[u] : -vp[u];
+                    }
+                }
             }
             __syncthreads();
             const int64_t lo = (a > p) ? a : p, hi = (b < p + cnt) ? b : p + cnt;
