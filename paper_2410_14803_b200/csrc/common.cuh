@@ -53,6 +53,7 @@ struct WorkspaceHeader {
     unsigned int qmin;   // batch minimum of sampled masses (sampler)
     unsigned int done;   // finished-block counter (sampler)
     unsigned int bad_epoch; // call number whose offsets failed validation (scan)
+    unsigned int left;      // blocks that have taken the batch minimum and are leaving (sampler)
 };
 constexpr size_t kHeaderBytes = 256;
 

@@ -111,6 +111,7 @@ __global__ void __launch_bounds__(256) build_leaf_kernel(Tree t, int vec_ok) {
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         t.hdr->qmin = 0xffffffffu;
         t.hdr->done = 0u;
+        t.hdr->left = 0u;
     }
     const int64_t g0 = (int64_t)blockIdx.x * kFan + warp * 4;
     unsigned long long s[4];
@@ -192,7 +193,7 @@ struct TopCache {
 
 __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     Tree t, TopCache tc, const unsigned long long *__restrict__ u, int64_t k, float beta, int normalise,
-    int64_t *__restrict__ idx_out, float *__restrict__ w_out, int vec_ok) {
+    int64_t *__restrict__ idx_out, float *__restrict__ w_out, int vec_ok, int together) {
     __shared__ __align__(128) unsigned long long s_top[kTopCap];
     __shared__ __align__(8) uint64_t s_bar;
     __shared__ int s_last;
@@ -224,6 +225,8 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
             }
         }
     }
+    uint32_t my_q = 0u; // mass of this warp's draw, in the lane that found it (`together` mode)
+    bool mine = false;
     if (j < k) {
         // top level: its entries sum to the total mass
         int l = t.levels;
@@ -265,7 +268,10 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
             if (idx >= t.n) { idx = t.n - 1; qs = 1u; set_status(&t.hdr->status, DISTRL_ERR_INDEX); }
             idx_out[j] = idx;
             if (w_out) {
-                if (normalise) {
+                if (normalise && together) {
+                    my_q = qs; // stays in the register until the batch minimum is known
+                    mine = true;
+                } else if (normalise) {
                     w_out[j] = __uint_as_float(qs); // parked here until the batch minimum is known
                 } else {
                     w_out[j] = powf((float)((double)t.n * (double)qs / (double)total), -beta);
@@ -274,6 +280,38 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
         }
     }
     if (!(w_out && normalise)) return;
+    if (together) {
+        // Every block of the grid is resident at once (the host checked that the grid fits), so the
+        // blocks can wait for one another: each adds its smallest mass to the batch minimum, counts
+        // itself in and polls the count; when it is complete the minimum is final and every draw is
+        // rescaled from its register.  The largest weight belongs to the smallest sampled mass, so
+        // w_j = (q_j / q_min)^-beta.  The wait is bounded; the last block to leave resets the words.
+        if (mine) atomicMin(&s_qmin, my_q);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            atomicMin(&t.hdr->qmin, s_qmin);
+            unsigned int seen;
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(seen) : "l"(&t.hdr->done) : "memory");
+            ++seen;
+            unsigned int spins = 0;
+            while (seen < gridDim.x) {
+                if (++spins > (1u << 22)) { set_status(&t.hdr->status, DISTRL_ERR_TIMEOUT); break; }
+                seen = ld_acquire_u32(&t.hdr->done);
+            }
+            s_qmin = __ldcg(&t.hdr->qmin);
+        }
+        __syncthreads();
+        if (mine) w_out[j] = powf((float)((double)my_q / (double)s_qmin), -beta);
+        if (threadIdx.x == 0) {
+            const unsigned int gone = atomicAdd(&t.hdr->left, 1u);
+            if (gone == gridDim.x - 1) { // everybody has read the minimum: ready for the next call
+                t.hdr->qmin = 0xffffffffu;
+                t.hdr->done = 0u;
+                t.hdr->left = 0u;
+            }
+        }
+        return;
+    }
     // The block that finishes last divides by the batch maximum.  The largest weight belongs to the
     // smallest sampled mass, so w_j = (q_j / q_min)^-beta; that block finds q_min among the parked
     // masses itself, so the other blocks pay a single atomic each.
@@ -646,10 +684,25 @@ extern "C" int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k
     if (!u_fix || !idx_out) return DISTRL_ERR_NULL;
     if (!aligned_to(u_fix, 8) || !aligned_to(idx_out, 8) || !aligned_to(is_weight_out, 4)) return DISTRL_ERR_ALIGN;
     const int64_t blocks = ceil_div(k * 32, kSampleThreads);
+    // blocks may wait for one another only if the whole grid is resident at once
+    static int resident[64] = {0};
+    int dev = 0;
+    DISTRL_CUDA_TRY(cudaGetDevice(&dev));
+    int fit = 0;
+    if (dev >= 0 && dev < 64) {
+        if (!resident[dev]) {
+            int per_sm = 0, sms = 0;
+            DISTRL_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sample_kernel, kSampleThreads, 0));
+            DISTRL_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+            resident[dev] = per_sm * sms > 0 ? per_sm * sms : -1;
+        }
+        fit = resident[dev];
+    }
+    const int together = (normalise && is_weight_out && fit > 0 && blocks <= fit) ? 1 : 0;
     DISTRL_CUDA_TRY(launch_pdl(sample_kernel, dim3((unsigned)blocks), dim3(kSampleThreads), 0,
                                static_cast<cudaStream_t>(stream), s->tree, s->top,
                                reinterpret_cast<const unsigned long long *>(u_fix), k, beta, normalise, idx_out,
-                               is_weight_out, s->vec_ok));
+                               is_weight_out, s->vec_ok, together));
     return DISTRL_OK;
 }
 
