@@ -211,6 +211,11 @@ int distrl_build_sampler(uint32_t *prio_q, int64_t n, void *workspace,
  *   is_weight_out : [k] fp32 or NULL: w_j = (n q_idx / total)^(-beta)
  *       (importance-sampling weight of prioritized replay, the definition the
  *       paper's replay cites); divided by the batch maximum if normalise != 0.
+ * A normalising call whose grid fits the GPU at once (a few thousand draws)
+ * lets its thread blocks wait for one another on the device for the batch
+ * maximum; the wait is bounded and reports DISTRL_ERR_TIMEOUT in the status
+ * word if another kernel holds the SMs for seconds.  Calls on one sampler must
+ * not overlap on the GPU (they share words of its workspace).
  */
 int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k, float beta,
                   int normalise, int64_t *idx_out, float *is_weight_out, void *stream);
