@@ -287,6 +287,14 @@ int distrl_destroy_sampler(distrl_sampler *s);
  * first device-side error recorded since the last read) and clears it. */
 int distrl_get_status(void *workspace, void *stream);
 
+/* Self-test of the library's bounded device-side waits (no counterpart in the
+ * paper): launches one warp that waits, with a limit of about a thousand polls,
+ * for a tile that nothing publishes.  Afterwards distrl_get_status(workspace)
+ * returns DISTRL_ERR_TIMEOUT; the kernel neither traps nor hangs.  Lets a caller
+ * check that its error handling sees device-side timeouts.
+ *   workspace : a retrace workspace (>= distrl_retrace_workspace_bytes(1024)). */
+int distrl_selftest_bounded_wait(void *workspace, size_t workspace_bytes, void *stream);
+
 const char *distrl_error_string(int code);
 const char *distrl_last_cuda_error(void); /* text of the last failed CUDA call, this thread */
 const char *distrl_version(void);

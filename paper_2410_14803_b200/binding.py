@@ -86,6 +86,7 @@ def _load():
         "distrl_sampler_level": (ci, [vp, ci, ctypes.POINTER(sz), ctypes.POINTER(i64)]),
         "distrl_destroy_sampler": (ci, [vp]),
         "distrl_get_status": (ci, [vp, vp]),
+        "distrl_selftest_bounded_wait": (ci, [vp, sz, vp]),
         "distrl_error_string": (ctypes.c_char_p, [ci]),
         "distrl_last_cuda_error": (ctypes.c_char_p, []),
         "distrl_version": (ctypes.c_char_p, []),
@@ -160,6 +161,11 @@ def distrl_sampler_workspace_bytes(n: int) -> int:
 def distrl_workspace_init(workspace: torch.Tensor, stream=None):
     _check(_load().distrl_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(),
                                          _stream(stream)), "distrl_workspace_init")
+
+
+def distrl_selftest_bounded_wait(workspace: torch.Tensor, stream=None):
+    _check(_load().distrl_selftest_bounded_wait(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                                _stream(stream)), "distrl_selftest_bounded_wait")
 
 
 def distrl_get_status(workspace: torch.Tensor, stream=None) -> int:

@@ -104,6 +104,20 @@ def test_retrace_bad_offsets_are_reported_not_fatal():
     check_retrace(np.array([0, 10, 20], dtype=np.int64), r, V, lp, lm, 0.9, 0.9)
 
 
+def test_a_wait_that_runs_out_is_reported_not_fatal():
+    # one warp waits, with a short limit, for a tile that nothing publishes: the status word must say so,
+    # and the same workspace must serve an ordinary call right after
+    n = 5000
+    ws = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws)
+    distrl.distrl_selftest_bounded_wait(ws)
+    assert distrl.distrl_get_status(ws) == distrl.binding.ERR_TIMEOUT
+    assert distrl.distrl_get_status(ws) == 0       # reading cleared it
+    off = synth.adversarial_offsets("long_mixed", n)
+    r, V, lp, lm = random_batch(5, off)
+    check_retrace(off, r, V, lp, lm, 0.99, 0.95)
+
+
 def test_mc_returns():
     for index in (1, 2):
         w = synth.make_workload(index)
