@@ -498,6 +498,31 @@ def test_token_level_bad_step_offsets_are_reported_not_fatal():
     assert good["status"] == 0
 
 
+def test_token_level_repeated_runs_agree_bit_for_bit():
+    # the token kernel's warps hand data to one another through shared-memory buffers guarded by
+    # mbarriers: ten runs on the same inputs and workspace must agree bit for bit
+    w = synth.make_workload(4, n_override=400001)
+    a = w.arrays
+    n = w.n
+    rng = np.random.default_rng(8)
+    t_off, t_r, t_V = dev(a["traj_offsets"]), dev(rng.normal(0, 1, n).astype(np.float32)), dev(rng.random(n, dtype=np.float32))
+    t_sto = dev(a["step_token_offsets"])
+    t_tp, t_tm = dev(a["tok_logp_target"], torch.bfloat16), dev(a["tok_logp_behaviour"], torch.bfloat16)
+    batch = distrl.make_batch(t_off, t_r, t_V, None, None, None, t_sto, t_tp, t_tm)
+    ws = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws)
+    first = None
+    for _ in range(10):
+        out = [torch.full((n,), float("nan"), dtype=torch.float32, device="cuda") for _ in range(5)]
+        distrl.distrl_retrace_targets(batch, w.gamma, w.lam, *out, workspace=ws)
+        got = [o.cpu().numpy().view(np.uint32) for o in out]
+        if first is None:
+            first = got
+        for g, f in zip(got, first):
+            np.testing.assert_array_equal(g, f)
+    assert distrl.distrl_get_status(ws) == 0
+
+
 def test_token_level_single_token_steps_equal_plain_logp():
     # one token per step: the token path must agree with the fp32-logp path on the same numbers
     n = 30000
