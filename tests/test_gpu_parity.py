@@ -498,29 +498,43 @@ def test_token_level_bad_step_offsets_are_reported_not_fatal():
     assert good["status"] == 0
 
 
-def test_token_level_repeated_runs_agree_bit_for_bit():
-    # the token kernel's warps hand data to one another through shared-memory buffers guarded by
-    # mbarriers: ten runs on the same inputs and workspace must agree bit for bit
-    w = synth.make_workload(4, n_override=400001)
-    a = w.arrays
-    n = w.n
+@pytest.mark.parametrize("pattern", ["workload", "alternating"])
+def test_token_level_repeated_runs_agree_bit_for_bit(pattern):
+    # The token kernel's warps hand data to one another through shared-memory buffers guarded by
+    # mbarriers, and drift apart by up to a tile: forty runs on the same inputs and workspace must
+    # agree bit for bit.  "alternating": tiles of one token per step alternate with tiles of 17, so
+    # that the same shared-memory positions belong to different warps in consecutive tiles.
+    if pattern == "workload":
+        w = synth.make_workload(4, n_override=1500001)
+        a = w.arrays
+        n, off, sto, tp, tm = w.n, a["traj_offsets"], a["step_token_offsets"], a["tok_logp_target"], a["tok_logp_behaviour"]
+    else:
+        n = 1200000
+        rng = np.random.default_rng(12)
+        cnt = np.where((np.arange(n) // 512) % 2 == 0, 1, 17)
+        sto = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int64)
+        nt = int(sto[-1])
+        tm = synth.f32_to_bf16_bits((rng.standard_normal(nt) * 0.3 - 0.3).astype(np.float32))
+        tp = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(tm) + (rng.standard_normal(nt) * 0.05).astype(np.float32))
+        off = synth.adversarial_offsets("long_mixed", n, tile=512)
     rng = np.random.default_rng(8)
-    t_off, t_r, t_V = dev(a["traj_offsets"]), dev(rng.normal(0, 1, n).astype(np.float32)), dev(rng.random(n, dtype=np.float32))
-    t_sto = dev(a["step_token_offsets"])
-    t_tp, t_tm = dev(a["tok_logp_target"], torch.bfloat16), dev(a["tok_logp_behaviour"], torch.bfloat16)
+    t_off, t_r, t_V = dev(off), dev(rng.normal(0, 1, n).astype(np.float32)), dev(rng.random(n, dtype=np.float32))
+    t_sto, t_tp, t_tm = dev(sto), dev(tp, torch.bfloat16), dev(tm, torch.bfloat16)
     batch = distrl.make_batch(t_off, t_r, t_V, None, None, None, t_sto, t_tp, t_tm)
     ws = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
     distrl.distrl_workspace_init(ws)
     first = None
-    for _ in range(10):
+    for _ in range(40):
         out = [torch.full((n,), float("nan"), dtype=torch.float32, device="cuda") for _ in range(5)]
-        distrl.distrl_retrace_targets(batch, w.gamma, w.lam, *out, workspace=ws)
-        got = [o.cpu().numpy().view(np.uint32) for o in out]
+        distrl.distrl_retrace_targets(batch, 0.99, 0.95, *out, workspace=ws)
+        got = [o.view(torch.int32) for o in out]
         if first is None:
             first = got
         for g, f in zip(got, first):
-            np.testing.assert_array_equal(g, f)
+            assert torch.equal(g, f)                  # compared on the device: bit patterns
     assert distrl.distrl_get_status(ws) == 0
+    lp = oracle.token_logp(sto, oracle.bf16_bits_to_f64(tp))
+    assert_close(first[3].view(torch.float32).cpu().numpy(), lp, "token logp_target")
 
 
 def test_token_level_single_token_steps_equal_plain_logp():
