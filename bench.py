@@ -484,13 +484,13 @@ def run_ours(args):
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the Retrace call's kernels, from the ncu captures
 # summarised under profiles/:
-#   "large": scan_pipe_kernel 270.59 + 153.01 MB and scan_mask_kernel 11.28 MB, captured at full size
+#   "large": scan_pipe_kernel 270.60 + 153.06 MB and scan_mask_kernel 11.28 MB, captured at full size
 #            (profiles/scan_pipe_kernel_large.md);
-#   "token": scan_tok_pipe_kernel 344.47 + 65.91 MB on a 4,194,304-step case of the same workload, scaled by 16 to
-#            the full 67,108,864 steps (every array grows in proportion), plus the 34.6 MB of trajectory offsets
-#            that scan_mask_kernel reads (profiles/scan_tok_pipe_kernel_token.md).
+#   "token": scan_tok_pipe_kernel 344.47 + 64.46 MB and scan_mask_kernel 2.19 MB on a 4,194,304-step case of the
+#            same workload, scaled by 16 to the full 67,108,864 steps (every array grows in proportion)
+#            (profiles/scan_tok_pipe_kernel_token.md).
 # Other workloads have no capture: reported as null.
-TRAFFIC_BYTES_PER_LAUNCH = {"large": 434_880_000, "token": None}   # token kernel changed since its capture
+TRAFFIC_BYTES_PER_LAUNCH = {"large": 434_940_000, "token": 16 * 411_120_000}
 
 
 def main():
