@@ -213,9 +213,12 @@ int distrl_build_sampler(uint32_t *prio_q, int64_t n, void *workspace,
  *       paper's replay cites); divided by the batch maximum if normalise != 0.
  * A normalising call whose grid fits the GPU at once (a few thousand draws)
  * lets its thread blocks wait for one another on the device for the batch
- * maximum; the wait is bounded and reports DISTRL_ERR_TIMEOUT in the status
- * word if another kernel holds the SMs for seconds.  Calls on one sampler must
- * not overlap on the GPU (they share words of its workspace).
+ * maximum; it is launched cooperatively, so the blocks are on the GPU together
+ * whatever else runs there (if that launch is refused the call takes the path
+ * of larger batches, where the last block does the rescaling).  The wait is
+ * bounded all the same and reports DISTRL_ERR_TIMEOUT in the status word.
+ * Calls on one sampler must not overlap on the GPU (they share words of its
+ * workspace); calls on different samplers may.
  */
 int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k, float beta,
                   int normalise, int64_t *idx_out, float *is_weight_out, void *stream);

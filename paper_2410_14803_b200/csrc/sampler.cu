@@ -699,10 +699,30 @@ extern "C" int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k
         fit = resident[dev];
     }
     const int together = (normalise && is_weight_out && fit > 0 && blocks <= fit) ? 1 : 0;
+    const unsigned long long *u64 = reinterpret_cast<const unsigned long long *>(u_fix);
+    if (together) {
+        // Blocks that wait for one another must all be on the GPU at the same time whatever else runs
+        // there (another stream's kernels, another sampler's draws): a cooperative launch guarantees
+        // that, or fails, in which case the call goes the other way below.
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)blocks);
+        cfg.blockDim = dim3(kSampleThreads);
+        cfg.stream = static_cast<cudaStream_t>(stream);
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeCooperative;
+        attr[1].val.cooperative = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        if (cudaLaunchKernelEx(&cfg, sample_kernel, s->tree, s->top, u64, k, beta, normalise, idx_out, is_weight_out,
+                               s->vec_ok, 1) == cudaSuccess)
+            return DISTRL_OK;
+        (void)cudaGetLastError(); // not launched: fall through to the launch that needs no co-residency
+    }
     DISTRL_CUDA_TRY(launch_pdl(sample_kernel, dim3((unsigned)blocks), dim3(kSampleThreads), 0,
-                               static_cast<cudaStream_t>(stream), s->tree, s->top,
-                               reinterpret_cast<const unsigned long long *>(u_fix), k, beta, normalise, idx_out,
-                               is_weight_out, s->vec_ok, together));
+                               static_cast<cudaStream_t>(stream), s->tree, s->top, u64, k, beta, normalise, idx_out,
+                               is_weight_out, s->vec_ok, 0));
     return DISTRL_OK;
 }
 

@@ -296,6 +296,36 @@ def test_sampler_build_and_sample(n, heavy):
     s.close()
 
 
+def test_two_samplers_drawing_at_the_same_time_on_two_streams():
+    # A normalising draw lets its blocks wait for one another; two such draws from different samplers
+    # on different streams must not starve each other (the launch is cooperative: each grid gets the
+    # SMs it needs at once, or waits as a whole).
+    k = 4096
+    qa, qb = _masses(1 << 20, 3), _masses((1 << 20) + 77, 4, heavy=False)
+    (sa, tqa, wsa), (sb, tqb, wsb) = _build(qa), _build(qb)
+    st_a, st_b = torch.cuda.Stream(), torch.cuda.Stream()
+    rng = np.random.default_rng(99)
+    torch.cuda.synchronize()
+    for rnd in range(25):
+        ua = rng.integers(0, 2 ** 64, size=k, dtype=np.uint64)
+        ub = rng.integers(0, 2 ** 64, size=k, dtype=np.uint64)
+        d_ua, d_ub = dev(ua.view(np.int64)), dev(ub.view(np.int64))
+        ia, ib = (torch.full((k,), -1, dtype=torch.int64, device="cuda") for _ in range(2))
+        wa, wb = (torch.full((k,), float("nan"), dtype=torch.float32, device="cuda") for _ in range(2))
+        torch.cuda.synchronize()
+        for _ in range(4):       # several draws in flight on each stream
+            distrl.distrl_sample(sa, d_ua, 0.4, True, ia, wa, stream=st_a)
+            distrl.distrl_sample(sb, d_ub, 0.6, True, ib, wb, stream=st_b)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(ia.cpu().numpy(), sample_by_prefix(qa, ua))
+        np.testing.assert_array_equal(ib.cpu().numpy(), sample_by_prefix(qb, ub))
+        assert_close(wa.cpu().numpy(), oracle.is_weights(qa, ia.cpu().numpy(), 0.4, True), "is_weight a")
+        assert_close(wb.cpu().numpy(), oracle.is_weights(qb, ib.cpu().numpy(), 0.6, True), "is_weight b")
+    assert distrl.distrl_get_status(wsa) == 0 and distrl.distrl_get_status(wsb) == 0
+    sa.close()
+    sb.close()
+
+
 def test_sampling_brute_force_on_device():
     # every threshold y in [0, total) must land on index i exactly q_i times
     q = np.array([3, 1, 7, 1, 1, 12, 5] * 40, dtype=np.uint32)
