@@ -54,6 +54,7 @@ struct WorkspaceHeader {
     unsigned int done;   // finished-block counter (sampler)
     unsigned int bad_epoch; // call number whose offsets failed validation (scan)
     unsigned int left;      // blocks that have taken the batch minimum and are leaving (sampler)
+    unsigned int tok_dense; // token-level scan: the steps own too many tokens on average for the pipelined kernel
 };
 constexpr size_t kHeaderBytes = 256;
 
