@@ -462,7 +462,7 @@ def run_ours(args):
             "priorities_gbs": prio_bytes / (stage_ms[1] * 1e-3) / 1e9,
             "build_sampler_gbs": build_bytes / (stage_ms[2] * 1e-3) / 1e9,
         },
-        "roofline": {"bound": "hbm", "kernel": ("scan_mask_kernel + scan_pipe_kernel<fused> (distrl_retrace_priorities_build)" if args.fused else "scan_mask_kernel + %s (distrl_retrace_targets)" % ("scan_tok_pipe_kernel" if tok else "scan_pipe_kernel")), "achieved": ach, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": ("scan_mask_kernel + scan_pipe_kernel<fused> (distrl_retrace_priorities_build)" if args.fused else "scan_mask_kernel + %s (distrl_retrace_targets)" % ("scan_tok_pipe_kernel (+ two stand-ins that return at once)" if tok else "scan_pipe_kernel")), "achieved": ach, "peak": peak,
                      "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
                      "frac_of_nominal_8000": ach / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name) if (args.n_override is None and not args.fused) else None,
                      "algorithmic_bytes": retrace_bytes},
@@ -486,11 +486,11 @@ def run_ours(args):
 # summarised under profiles/:
 #   "large": scan_pipe_kernel 270.60 + 153.06 MB and scan_mask_kernel 11.28 MB, captured at full size
 #            (profiles/scan_pipe_kernel_large.md);
-#   "token": scan_tok_pipe_kernel 344.47 + 64.46 MB and scan_mask_kernel 2.19 MB on a 4,194,304-step case of the
-#            same workload, scaled by 16 to the full 67,108,864 steps (every array grows in proportion)
-#            (profiles/scan_tok_pipe_kernel_token.md).
+#   "token": scan_tok_pipe_kernel 344.47 + 63.74 MB, scan_mask_kernel 2.19 MB and the two stand-ins that return at
+#            once 0.06 MB on a 4,194,304-step case of the same workload, scaled by 16 to the full 67,108,864 steps
+#            (every array grows in proportion) (profiles/scan_tok_pipe_kernel_token.md).
 # Other workloads have no capture: reported as null.
-TRAFFIC_BYTES_PER_LAUNCH = {"large": 434_940_000, "token": 16 * 411_120_000}
+TRAFFIC_BYTES_PER_LAUNCH = {"large": 434_940_000, "token": 16 * 410_460_000}
 
 
 def main():
