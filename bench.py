@@ -258,7 +258,8 @@ def run_ours(args):
     ev = lambda: torch.cuda.Event(enable_timing=True)
     # a refresh of up to 8192 positions is one launch, a longer one a claim and an apply launch per 65536 positions
     per_round = 1 + (1 if (k <= 8192 and n < 2 ** 31) else 2 * ((k + 65535) // 65536))
-    launches_per_step = 2 + 1 + 2 + per_round * R   # end mask + scan, priorities, 2 build, (sample, refresh) x R
+    retrace_launches = 4 if tok else 2   # end mask + scan (token-level: + the two stand-ins for dense buffers)
+    launches_per_step = retrace_launches + 1 + 2 + per_round * R   # Retrace, priorities, 2 build, (sample, refresh) x R
     if args.fused:
         launches_per_step = 3 + per_round * R       # end mask + fused scan + upper tree levels, then the rounds
 
