@@ -509,6 +509,21 @@ def test_token_level_staging_corners(counts):
     _token_case(off, sto, tok_p, tok_m, 5)
 
 
+@pytest.mark.parametrize("lo,hi", [(20, 33), (17, 19), (16, 18)])
+def test_token_level_dense_buffers(lo, hi):
+    # mean token counts around and above what a stage of the pipelined kernel holds (about 17 per step):
+    # the call hands dense buffers to the general kernel; either way the results are the oracle's
+    n = 120001
+    rng = np.random.default_rng(lo * 100 + hi)
+    cnt = rng.integers(lo, hi, n)
+    sto = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int64)
+    nt = int(sto[-1])
+    tok_m = synth.f32_to_bf16_bits((rng.standard_normal(nt) * 0.3 - 0.3).astype(np.float32) / np.float32(2))
+    tok_p = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(tok_m) + (rng.standard_normal(nt) * 0.05).astype(np.float32))
+    off = synth.adversarial_offsets("long_mixed", n, tile=512)
+    _token_case(off, sto, tok_p, tok_m, 11)
+
+
 def test_token_level_bad_step_offsets_are_reported_not_fatal():
     n = 3000
     rng = np.random.default_rng(3)
