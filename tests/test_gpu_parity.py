@@ -64,6 +64,63 @@ def test_retrace_bootstrap_values():
     check_retrace(off, r, V, lp, lm, 0.97, 0.9, boot=boot)
 
 
+@pytest.mark.parametrize("kind", ["with_empty", "long_mixed", "ones", "tile_aligned", "tile_straddle", "single"])
+@pytest.mark.parametrize("n", [1, 129, 2047, 2048, 2049, 2176, 2177, 100003, 700001])
+def test_retrace_bootstrap_values_layouts(kind, n):
+    # bootstrap values with aligned arrays go through the pipelined kernel: ends inside the 128-item halo
+    # of a tile, on tile boundaries, empty trajectories in between, buffers shorter than a halo
+    off = synth.adversarial_offsets(kind, n)
+    r, V, lp, lm = random_batch(n + 7, off)
+    boot = np.random.default_rng(n).normal(0, 2, off.shape[0] - 1).astype(np.float32)
+    check_retrace(off, r, V, lp, lm, 0.97, 0.9, boot=boot)
+
+
+def test_retrace_bootstrap_values_through_the_general_kernel():
+    # arrays that are not 16-byte aligned; and a workspace without room for what the pipelined kernel
+    # keeps of the bootstrap values (the fixed array of the workspace-free entry point is one)
+    off = synth.adversarial_offsets("long_mixed", 50001)
+    r, V, lp, lm = random_batch(9, off)
+    boot = np.random.default_rng(5).normal(0, 2, off.shape[0] - 1).astype(np.float32)
+    check_retrace(off, r, V, lp, lm, 0.97, 0.9, boot=boot, misalign=True)
+    n = r.shape[0]
+    t = [dev(off), dev(r), dev(V), dev(lp), dev(lm), dev(boot)]     # kept alive: the batch only holds pointers
+    batch = distrl.make_batch(*t)
+    out = [torch.full((n,), float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
+    status = torch.full((1,), -77, dtype=torch.int32, device="cuda")
+    distrl.distrl_retrace_targets_static(batch, 0.97, 0.9, *out, status_out=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    vt, adv, dl = oracle.retrace(off, r, V, lp, lm, 0.97, 0.9, bootstrap=boot)
+    assert_close(out[0].cpu().numpy(), vt, "v_target")
+    assert_close(out[1].cpu().numpy(), adv, "advantage")
+    assert_close(out[2].cpu().numpy(), dl, "td_delta")
+
+
+def test_retrace_bootstrap_repeated_runs_agree_bit_for_bit():
+    n = 500001
+    off = synth.adversarial_offsets("long_mixed", n)
+    r, V, lp, lm = random_batch(77, off)
+    boot = np.random.default_rng(6).normal(0, 2, off.shape[0] - 1).astype(np.float32)
+    t = [dev(off), dev(r), dev(V), dev(lp), dev(lm), dev(boot)]
+    batch = distrl.make_batch(*t)
+    ws = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws)
+    first = None
+    for _ in range(20):
+        out = [torch.full((n,), float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
+        distrl.distrl_retrace_targets(batch, 0.99, 0.95, *out, workspace=ws)
+        got = [o.view(torch.int32) for o in out]
+        if first is None:
+            first = got
+        for g, f in zip(got, first):
+            assert torch.equal(g, f)
+    assert distrl.distrl_get_status(ws) == 0
+    vt, adv, dl = oracle.retrace(off, r, V, lp, lm, 0.99, 0.95, bootstrap=boot)
+    assert_close(first[0].view(torch.float32).cpu().numpy(), vt, "v_target")
+    assert_close(first[1].view(torch.float32).cpu().numpy(), adv, "advantage")
+    assert_close(first[2].view(torch.float32).cpu().numpy(), dl, "td_delta")
+
+
 @pytest.mark.parametrize("n", [3, 4099, 30011])
 def test_retrace_unaligned_pointers_and_ragged_tail(n):
     off = synth.adversarial_offsets("long_mixed", n)
