@@ -487,11 +487,11 @@ def run_ours(args):
 # summarised under profiles/:
 #   "large": scan_pipe_kernel 270.60 + 152.89 MB and scan_mask_kernel 11.28 MB, captured at full size
 #            (profiles/scan_pipe_kernel_large.md);
-#   "token": scan_tok_pipe_kernel 344.47 + 63.74 MB, scan_mask_kernel 2.19 MB and the two stand-ins that return at
+#   "token": scan_tok_pipe_kernel 344.49 + 64.17 MB, scan_mask_kernel 2.19 MB and the two stand-ins that return at
 #            once 0.06 MB on a 4,194,304-step case of the same workload, scaled by 16 to the full 67,108,864 steps
 #            (every array grows in proportion) (profiles/scan_tok_pipe_kernel_token.md).
 # Other workloads have no capture: reported as null.
-TRAFFIC_BYTES_PER_LAUNCH = {"large": 434_770_000, "token": 16 * 410_460_000}
+TRAFFIC_BYTES_PER_LAUNCH = {"large": 434_770_000, "token": 16 * 410_910_000}
 
 
 def main():
