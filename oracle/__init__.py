@@ -203,3 +203,29 @@ def replay_overwrite(q, head, new_q):
     lib = _load()
     lib.oracle_replay_overwrite.restype = ctypes.c_int64
     return int(lib.oracle_replay_overwrite(_n(q.shape[0]), _p(q), _n(head), _n(nq.shape[0]), _p(nq)))
+
+
+def actor_coefficients(logp_pi, logp_mu, advantage, idx=None, is_weight=None):
+    """w_j * rho_i * A_i for the sampled transitions (actor loss of Section 5.1 / App. A)."""
+    lp, lm, adv = _f64(logp_pi), _f64(logp_mu), _f64(advantage)
+    n = lp.shape[0]
+    ix = None if idx is None else _i64(idx)
+    k = n if ix is None else ix.shape[0]
+    w = _f64(is_weight)
+    out = np.empty(k, dtype=np.float64)
+    rc = _load().oracle_actor_coefficients(_n(n), _n(k), _p(ix), _p(lp), _p(lm), _p(adv), _p(w), _p(out))
+    if rc:
+        raise IndexError("index outside [0, n)")
+    return out
+
+
+def trajectory_ranges(traj_offsets, idx):
+    """[begin, end) of the flat buffer for each drawn trajectory index (Section 5.3)."""
+    off, ix = _i64(traj_offsets), _i64(idx)
+    k = ix.shape[0]
+    b = np.empty(k, dtype=np.int64)
+    e = np.empty(k, dtype=np.int64)
+    rc = _load().oracle_trajectory_ranges(_n(off.shape[0] - 1), _p(off), _n(k), _p(ix), _p(b), _p(e))
+    if rc:
+        raise IndexError("trajectory index outside [0, m)")
+    return b, e

@@ -299,3 +299,35 @@ int64_t oracle_replay_overwrite(int64_t n, uint32_t *q, int64_t head, int64_t k,
     }
     return i;
 }
+
+/* ------------------------------------------------------------------------- *
+ * Per-sample coefficient of the actor loss (Section 5.1, the policy loss, and App. A "Policy Update
+ * Mechanism"): the update direction is  - E_mu[ rho_t A(s_t,a_t) grad log pi(a_t|s_t) ],  so a
+ * sampled transition i enters with the scalar  rho_i A_i,  rho_i = pi(a_i|s_i) / mu(a_i|s_i),
+ * times its importance-sampling weight w_j when the batch was drawn by priority.
+ *   idx NULL : j runs over the k = n transitions in order;  w NULL : weight 1.
+ * ------------------------------------------------------------------------- */
+int oracle_actor_coefficients(int64_t n, int64_t k, const int64_t *idx, const double *lp,
+                              const double *lm, const double *adv, const double *w, double *coef)
+{
+    for (int64_t j = 0; j < k; ++j) {
+        int64_t i = idx ? idx[j] : j;
+        if (i < 0 || i >= n) return -1;
+        double rho = exp(lp[i] - lm[i]);
+        coef[j] = (w ? w[j] : 1.0) * rho * adv[i];
+    }
+    return 0;
+}
+
+/* Trajectory-level sampling (Section 5.3 prioritises trajectories tau): a drawn trajectory index j
+ * stands for the transitions [off[j], off[j+1]) of the flat buffer. */
+int oracle_trajectory_ranges(int64_t m, const int64_t *off, int64_t k, const int64_t *idx,
+                             int64_t *begin, int64_t *end)
+{
+    for (int64_t j = 0; j < k; ++j) {
+        if (idx[j] < 0 || idx[j] >= m) return -1;
+        begin[j] = off[idx[j]];
+        end[j] = off[idx[j] + 1];
+    }
+    return 0;
+}

@@ -51,6 +51,14 @@ MUTATIONS = {
         ("g = r[t] + gamma * g;", "g = r[t] + g;"),
     "circular overwrite does not wrap":
         ("i = (i + 1) % n;", "i = (i + 1 < n) ? i + 1 : i;"),
+    "actor coefficient: ratio inverted":
+        ("double rho = exp(lp[i] - lm[i]);\n        coef[j]", "double rho = exp(lm[i] - lp[i]);\n        coef[j]"),
+    "actor coefficient: importance-sampling weight dropped":
+        ("coef[j] = (w ? w[j] : 1.0) * rho * adv[i];", "coef[j] = rho * adv[i];"),
+    "actor coefficient: advantage read at the batch position instead of the drawn index":
+        ("coef[j] = (w ? w[j] : 1.0) * rho * adv[i];", "coef[j] = (w ? w[j] : 1.0) * rho * adv[j];"),
+    "trajectory range ends at its own start offset":
+        ("end[j] = off[idx[j] + 1];", "end[j] = off[idx[j]];"),
 }
 
 

@@ -368,3 +368,51 @@ def test_circular_overwrite_wraps_and_later_writes_win():
     q = np.arange(1, 4, dtype=np.uint32)                      # more writes than slots: the last three survive
     nxt = oracle.replay_overwrite(q, 1, np.arange(10, 18, dtype=np.uint32))
     assert q.tolist() == [15, 16, 17] and nxt == 0            # slots visited 1,2,0,1,2,0,1,2
+
+
+# ------------------------------------------------ actor-loss coefficients ---
+def test_actor_coefficient_hand_case_and_on_policy():
+    # pi = 0.5, mu = 0.25 -> rho = 2; A = 3; w = 0.5  ->  0.5 * 2 * 3 = 3
+    c = oracle.actor_coefficients([math.log(0.5)], [math.log(0.25)], [3.0], idx=[0], is_weight=[0.5])
+    assert c[0] == pytest.approx(3.0, rel=1e-15)
+    rng = np.random.default_rng(5)
+    lm = rng.normal(-4, 2, 300)
+    A = rng.normal(0, 1, 300)
+    np.testing.assert_array_equal(oracle.actor_coefficients(lm, lm, A), A)   # on-policy: rho = 1
+
+
+def test_actor_coefficient_is_the_derivative_of_the_importance_weighted_surrogate():
+    # grad_theta [ w * (pi_theta / mu) * A ] = w * rho * A * grad_theta log pi_theta, so the coefficient
+    # equals d/d(log pi) of S = w * A * exp(log pi - log mu): central differences, independent numpy.
+    rng = np.random.default_rng(6)
+    n, k = 500, 64
+    lm = rng.normal(-5, 2, n)
+    lp = lm + rng.normal(0, 0.7, n)
+    A = rng.normal(0, 2, n)
+    idx = rng.integers(0, n, k)
+    w = rng.uniform(0.05, 1.0, k)
+    h = 1e-6
+    S = lambda x: w * A[idx] * np.exp(x - lm[idx])
+    fd = (S(lp[idx] + h) - S(lp[idx] - h)) / (2 * h)
+    np.testing.assert_allclose(oracle.actor_coefficients(lp, lm, A, idx, w), fd, rtol=1e-8, atol=1e-9)
+    # swapping the two policies inverts the ratio
+    a = oracle.actor_coefficients(lp, lm, np.ones(n))
+    b = oracle.actor_coefficients(lm, lp, np.ones(n))
+    np.testing.assert_allclose(a * b, np.ones(n), rtol=1e-14)
+    with pytest.raises(IndexError):
+        oracle.actor_coefficients(lp, lm, A, idx=[n])
+
+
+def test_trajectory_ranges_tile_the_buffer():
+    rng = np.random.default_rng(8)
+    off = np.concatenate([[0], np.cumsum(rng.integers(0, 9, 40))]).astype(np.int64)
+    b, e = oracle.trajectory_ranges(off, np.arange(40))
+    assert b[0] == 0 and e[-1] == off[-1]
+    np.testing.assert_array_equal(b[1:], e[:-1])                      # consecutive, no gaps
+    np.testing.assert_array_equal(e - b, np.diff(off))                # lengths
+    pick = rng.integers(0, 40, 17)
+    pb, pe = oracle.trajectory_ranges(off, pick)
+    for j, t in enumerate(pick):
+        assert (pb[j], pe[j]) == (off[t], off[t + 1])
+    with pytest.raises(IndexError):
+        oracle.trajectory_ranges(off, [40])
