@@ -275,6 +275,38 @@ int distrl_retrace_priorities_build(const distrl_batch *batch, float gamma, floa
                                     void *sampler_workspace, size_t sampler_workspace_bytes,
                                     void *stream, distrl_sampler **out);
 
+/*
+ * What a drawn batch carries into the actor loss (Section 5.1, the policy loss;
+ * App. A "Policy Update Mechanism"): the update direction is
+ * -E_mu[rho_t A(s_t,a_t) grad log pi(a_t|s_t)], so sampled transition i = idx[j]
+ * enters with the scalar
+ *   coef[j] = is_weight[j] * rho_i * A_i,   rho_i = exp(logp_target[i] - logp_behaviour[i]).
+ *   idx       : [k] device indices into the buffer (e.g. from distrl_sample), or
+ *               NULL with k == n for the whole buffer in order.
+ *   advantage : [n], e.g. the output of distrl_retrace_targets.
+ *   is_weight : [k] importance-sampling weights from distrl_sample, or NULL (= 1).
+ *   coef      : [k] output.
+ *   status_out_device : device int or NULL; set to DISTRL_ERR_INDEX if some
+ *               idx[j] lies outside [0, n) (that coef[j] is then NaN; nothing is
+ *               read out of bounds).
+ * fp32 arithmetic: one expf, two multiplies.
+ */
+int distrl_actor_coefficients(int64_t n, const int64_t *idx, int64_t k, const float *logp_target,
+                              const float *logp_behaviour, const float *advantage,
+                              const float *is_weight, float *coef, int *status_out_device,
+                              void *stream);
+
+/*
+ * Trajectory-level draws (Section 5.3 prioritises trajectories): with a sampler
+ * built over the M masses of distrl_compute_priorities_traj, a drawn index
+ * idx[j] stands for the transitions [begin[j], end[j]) =
+ * [traj_offsets[idx[j]], traj_offsets[idx[j]+1]) of the flat buffer.
+ *   idx outside [0, m): begin = end = -1 and *status_out_device (if given) is set
+ *   to DISTRL_ERR_INDEX.
+ */
+int distrl_trajectory_ranges(int64_t m, const int64_t *traj_offsets, const int64_t *idx, int64_t k,
+                             int64_t *begin, int64_t *end, int *status_out_device, void *stream);
+
 /* Writes total = sum_i q_i to *total_out_device (a device uint64). */
 int distrl_sampler_total(distrl_sampler *s, uint64_t *total_out_device, void *stream);
 

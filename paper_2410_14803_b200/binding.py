@@ -82,6 +82,8 @@ def _load():
                                                  ctypes.POINTER(distrl_prio_cfg), vp, vp, vp, vp, vp, vp, sz, vp, sz, vp,
                                                  ctypes.POINTER(vp)]),
         "distrl_replay_overwrite": (ci, [vp, i64, i64, vp, vp]),
+        "distrl_actor_coefficients": (ci, [i64, vp, i64, vp, vp, vp, vp, vp, vp, vp]),
+        "distrl_trajectory_ranges": (ci, [i64, vp, vp, i64, vp, vp, vp, vp]),
         "distrl_sampler_total": (ci, [vp, vp, vp]),
         "distrl_sampler_level": (ci, [vp, ci, ctypes.POINTER(sz), ctypes.POINTER(i64)]),
         "distrl_destroy_sampler": (ci, [vp]),
@@ -288,6 +290,37 @@ def distrl_replay_overwrite(s: Sampler, head: int, new_q: torch.Tensor, stream=N
         raise ValueError("new_q must hold 32-bit masses")
     _check(_load().distrl_replay_overwrite(s.handle, head, new_q.numel(), _ptr(new_q), _stream(stream)),
            "distrl_replay_overwrite")
+
+
+def distrl_actor_coefficients(logp_target: torch.Tensor, logp_behaviour: torch.Tensor, advantage: torch.Tensor,
+                              coef: torch.Tensor, idx: Optional[torch.Tensor] = None,
+                              is_weight: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+                              stream=None):
+    """coef[j] = is_weight[j] * rho_i * A_i for i = idx[j] (idx None: the whole buffer in order)."""
+    n = logp_target.numel()
+    k = n if idx is None else idx.numel()
+    for t in (logp_behaviour, advantage):
+        if t.numel() != n:
+            raise ValueError("per-transition arrays must have one length")
+    if coef.numel() != k or (is_weight is not None and is_weight.numel() != k):
+        raise ValueError("coef and is_weight must have one entry per batch position")
+    _check(_load().distrl_actor_coefficients(n, _ptr(idx, torch.int64), k, _ptr(logp_target, torch.float32),
+                                             _ptr(logp_behaviour, torch.float32), _ptr(advantage, torch.float32),
+                                             _ptr(is_weight, torch.float32), _ptr(coef, torch.float32),
+                                             _ptr(status, torch.int32), _stream(stream)),
+           "distrl_actor_coefficients")
+
+
+def distrl_trajectory_ranges(traj_offsets: torch.Tensor, idx: torch.Tensor, begin: torch.Tensor, end: torch.Tensor,
+                             status: Optional[torch.Tensor] = None, stream=None):
+    """[begin, end) of the flat buffer for each drawn trajectory index."""
+    k = idx.numel()
+    if begin.numel() != k or end.numel() != k:
+        raise ValueError("begin and end must have one entry per drawn index")
+    _check(_load().distrl_trajectory_ranges(traj_offsets.numel() - 1, _ptr(traj_offsets, torch.int64),
+                                            _ptr(idx, torch.int64), k, _ptr(begin, torch.int64),
+                                            _ptr(end, torch.int64), _ptr(status, torch.int32), _stream(stream)),
+           "distrl_trajectory_ranges")
 
 
 def distrl_sampler_total(s: Sampler, total_out: torch.Tensor, stream=None):

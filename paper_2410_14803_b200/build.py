@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libdistrl_b200.so")
-SOURCES = ["api.cu", "retrace.cu", "priority.cu", "sampler.cu"]
+SOURCES = ["api.cu", "retrace.cu", "priority.cu", "sampler.cu", "batch.cu"]
 
 
 def _newest_source_mtime() -> float:

@@ -1,0 +1,133 @@
+// What the learner takes from a drawn batch: the scalar each transition carries into the actor
+// loss of Section 5.1 (w_j * rho_i * A_i), and, for trajectory-level draws (Section 5.3), the
+// transition range a trajectory index stands for.  Both are gathers or plain streams: no
+// dependency between outputs, so the kernels are sized for coalescing and loads in flight only.
+#include "common.cuh"
+
+#include <cmath>
+
+namespace distrl {
+
+constexpr int kBatchThreads = 256;
+
+__device__ __forceinline__ float actor_term(float lp, float lm, float adv) { return expf(lp - lm) * adv; }
+
+// Whole buffer in order: 12 bytes in, 4 out per transition.
+template <bool VEC>
+__global__ void __launch_bounds__(kBatchThreads) actor_stream_kernel(
+    int64_t n, const float *__restrict__ lp, const float *__restrict__ lm, const float *__restrict__ adv,
+    const float *__restrict__ w, float *__restrict__ coef) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (VEC) {
+        const int64_t n4 = n >> 2;
+        for (int64_t v = g; v < n4; v += stride) {
+            const float4 p = ldg_stream_f4(lp + 4 * v), m = ldg_stream_f4(lm + 4 * v), a = ldg_stream_f4(adv + 4 * v);
+            float4 c = make_float4(actor_term(p.x, m.x, a.x), actor_term(p.y, m.y, a.y),
+                                   actor_term(p.z, m.z, a.z), actor_term(p.w, m.w, a.w));
+            if (w) {
+                const float4 ww = ldg_stream_f4(w + 4 * v);
+                c = make_float4(ww.x * c.x, ww.y * c.y, ww.z * c.z, ww.w * c.w);
+            }
+            stg_stream_f4(coef + 4 * v, c);
+        }
+        for (int64_t t = 4 * n4 + g; t < n; t += stride) {
+            const float c = actor_term(lp[t], lm[t], adv[t]);
+            coef[t] = w ? w[t] * c : c;
+        }
+    } else {
+        for (int64_t t = g; t < n; t += stride) {
+            const float c = actor_term(lp[t], lm[t], adv[t]);
+            coef[t] = w ? w[t] * c : c;
+        }
+    }
+}
+
+// Drawn batch: one thread per batch position, three independent 4-byte gathers each.
+__global__ void __launch_bounds__(kBatchThreads) actor_gather_kernel(
+    int64_t n, int64_t k, const int64_t *__restrict__ idx, const float *__restrict__ lp,
+    const float *__restrict__ lm, const float *__restrict__ adv, const float *__restrict__ w,
+    float *__restrict__ coef, int *status) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k; j += stride) {
+        const int64_t i = idx[j];
+        if (i < 0 || i >= n) {
+            if (status) set_status(status, DISTRL_ERR_INDEX);
+            coef[j] = nanf("");
+            continue;
+        }
+        const float c = actor_term(lp[i], lm[i], adv[i]);
+        coef[j] = w ? w[j] * c : c;
+    }
+}
+
+__global__ void __launch_bounds__(kBatchThreads) traj_ranges_kernel(
+    int64_t m, const int64_t *__restrict__ off, int64_t k, const int64_t *__restrict__ idx,
+    int64_t *__restrict__ begin, int64_t *__restrict__ end, int *status) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k; j += stride) {
+        const int64_t t = idx[j];
+        if (t < 0 || t >= m) {
+            if (status) set_status(status, DISTRL_ERR_INDEX);
+            begin[j] = -1;
+            end[j] = -1;
+            continue;
+        }
+        begin[j] = off[t];
+        end[j] = off[t + 1];
+    }
+}
+
+static int batch_grid(int64_t items) {
+    int64_t b = ceil_div(items, kBatchThreads);
+    if (b < 1) b = 1;
+    const int64_t cap = 148 * 8; // 148 SMs x 8 resident blocks of 256 threads
+    return (int)(b > cap ? cap : b);
+}
+
+} // namespace distrl
+
+using namespace distrl;
+
+extern "C" int distrl_actor_coefficients(int64_t n, const int64_t *idx, int64_t k, const float *logp_target,
+                                         const float *logp_behaviour, const float *advantage,
+                                         const float *is_weight, float *coef, int *status_out_device,
+                                         void *stream) {
+    if (n < 0 || n > DISTRL_MAX_N || k < 0 || k > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
+    if (!idx && k != n) return DISTRL_ERR_SIZE;
+    if (k == 0) return DISTRL_OK;
+    if (!logp_target || !logp_behaviour || !advantage || !coef) return DISTRL_ERR_NULL;
+    const void *ptrs[] = {logp_target, logp_behaviour, advantage, is_weight, coef, status_out_device};
+    bool vec = true;
+    for (const void *p : ptrs) {
+        if (p && !aligned_to(p, 4)) return DISTRL_ERR_ALIGN;
+        if (p && p != status_out_device && !aligned_to(p, 16)) vec = false;
+    }
+    if (idx && !aligned_to(idx, 8)) return DISTRL_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (idx)
+        actor_gather_kernel<<<batch_grid(k), kBatchThreads, 0, st>>>(n, k, idx, logp_target, logp_behaviour,
+                                                                     advantage, is_weight, coef, status_out_device);
+    else if (vec)
+        actor_stream_kernel<true><<<batch_grid(n / 4 + 1), kBatchThreads, 0, st>>>(n, logp_target, logp_behaviour,
+                                                                                   advantage, is_weight, coef);
+    else
+        actor_stream_kernel<false><<<batch_grid(n), kBatchThreads, 0, st>>>(n, logp_target, logp_behaviour,
+                                                                            advantage, is_weight, coef);
+    DISTRL_CUDA_TRY(cudaGetLastError());
+    return DISTRL_OK;
+}
+
+extern "C" int distrl_trajectory_ranges(int64_t m, const int64_t *traj_offsets, const int64_t *idx, int64_t k,
+                                        int64_t *begin, int64_t *end, int *status_out_device, void *stream) {
+    if (m < 0 || m > DISTRL_MAX_N || k < 0 || k > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
+    if (k == 0) return DISTRL_OK;
+    if (!traj_offsets || !idx || !begin || !end) return DISTRL_ERR_NULL;
+    if (!aligned_to(traj_offsets, 8) || !aligned_to(idx, 8) || !aligned_to(begin, 8) || !aligned_to(end, 8) ||
+        (status_out_device && !aligned_to(status_out_device, 4)))
+        return DISTRL_ERR_ALIGN;
+    traj_ranges_kernel<<<batch_grid(k), kBatchThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        m, traj_offsets, k, idx, begin, end, status_out_device);
+    DISTRL_CUDA_TRY(cudaGetLastError());
+    return DISTRL_OK;
+}

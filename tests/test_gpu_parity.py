@@ -861,3 +861,112 @@ def test_rounds_replayed_from_a_cuda_graph_match_the_oracle():
     assert distrl.distrl_get_status(ws) == 0
     del q1
     s.close()
+
+
+# ------------------------------------------------- what a drawn batch carries ---
+
+def _policy_arrays(n, seed):
+    rng = np.random.default_rng(seed)
+    lm = rng.normal(-5, 2, n).astype(np.float32)
+    lp = (lm + rng.normal(0, 0.7, n)).astype(np.float32)
+    adv = rng.normal(0, 2, n).astype(np.float32)
+    return lp, lm, adv
+
+
+@pytest.mark.parametrize("n", [1, 3, 4, 1023, 1024, 1025, 303_107, (1 << 21) + 3])
+@pytest.mark.parametrize("weights", [False, True])
+@pytest.mark.parametrize("misalign", [False, True])
+def test_actor_coefficients_whole_buffer(n, weights, misalign):
+    from helpers import dev_misaligned
+    up = dev_misaligned if misalign else dev
+    lp, lm, adv = _policy_arrays(n, n)
+    w = np.random.default_rng(n + 1).uniform(0.01, 1.0, n).astype(np.float32) if weights else None
+    coef = torch.full((n + 1,), float("nan"), dtype=torch.float32, device="cuda")
+    out = coef[1:] if misalign else coef[:n]
+    distrl.distrl_actor_coefficients(up(lp), up(lm), up(adv), out, is_weight=up(w) if weights else None)
+    torch.cuda.synchronize()
+    assert_close(out.cpu().numpy(), oracle.actor_coefficients(lp, lm, adv, None, w), "actor coefficient", tol=1e-5)
+    if not misalign:
+        assert np.isnan(coef[n].item())                                   # nothing written past the end
+
+
+@pytest.mark.parametrize("index", [1, 2])
+def test_actor_coefficients_of_a_prioritised_draw(index):
+    # the whole chain: Retrace advantages -> priorities -> draw -> coefficients of the drawn batch
+    w = synth.make_workload(index)
+    a = w.arrays
+    g = gpu_retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"], w.gamma, w.lam)
+    adv = g["advantage"]
+    mass, q = _gpu_priorities(w, g["td_delta"])
+    s, tq, ws = _build(q)
+    u = synth.uniforms(w, 0)
+    idx, wts = _sample(s, u, w.beta)
+    coef = torch.full((idx.shape[0],), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    distrl.distrl_actor_coefficients(dev(a["logp_target"]), dev(a["logp_behaviour"]), dev(adv), coef, idx=dev(idx),
+                                     is_weight=dev(wts), status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    ref = oracle.actor_coefficients(a["logp_target"], a["logp_behaviour"], adv, idx, wts)
+    assert_close(coef.cpu().numpy(), ref, "actor coefficient of the batch", tol=1e-5)
+    s.close()
+
+
+def test_actor_coefficients_edges():
+    lp, lm, adv = _policy_arrays(100, 3)
+    t = [dev(lp), dev(lm), dev(adv)]
+    # empty batch: nothing launched, nothing written
+    distrl.distrl_actor_coefficients(*t, torch.empty(0, dtype=torch.float32, device="cuda"),
+                                     idx=torch.empty(0, dtype=torch.int64, device="cuda"))
+    # indices outside the buffer: flagged, NaN, neighbours untouched and correct
+    idx = np.array([5, -1, 99, 100, 0, 1 << 40], dtype=np.int64)
+    coef = torch.zeros(idx.shape[0], dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    distrl.distrl_actor_coefficients(*t, coef, idx=dev(idx), status=status)
+    torch.cuda.synchronize()
+    c = coef.cpu().numpy()
+    good = np.array([0, 2, 4])
+    assert np.all(np.isnan(c[[1, 3, 5]]))
+    assert_close(c[good], oracle.actor_coefficients(lp, lm, adv, idx[good]), "in-range entries", tol=1e-5)
+    assert distrl.distrl_error_string(int(status.item())) == "index outside [0, n)"
+    # whole-buffer form needs k == n; required pointers are checked on the host
+    from paper_2410_14803_b200 import binding
+    lib = binding._load()
+    p = [x.data_ptr() for x in t]
+    assert lib.distrl_actor_coefficients(100, None, 7, p[0], p[1], p[2], None, coef.data_ptr(), None, None) == binding.ERR_SIZE
+    assert lib.distrl_actor_coefficients(100, None, 100, p[0], None, p[2], None, coef.data_ptr(), None, None) == binding.ERR_NULL
+    assert lib.distrl_actor_coefficients(100, None, 100, p[0], p[1] + 2, p[2], None, coef.data_ptr(), None, None) == binding.ERR_ALIGN
+
+
+def test_trajectory_level_draw_returns_transition_ranges():
+    w = synth.make_workload(1)
+    a = w.arrays
+    off = np.sort(np.concatenate([a["traj_offsets"], a["traj_offsets"][[7, 7, 300]]]))   # with empty trajectories
+    m = off.shape[0] - 1
+    delta = np.random.default_rng(4).normal(0, 1, w.n).astype(np.float32)
+    q = torch.empty(m, dtype=torch.int32, device="cuda")
+    distrl.distrl_compute_priorities_traj(dev(off), dev(delta), dev(a["logp_target"]), dev(a["logp_behaviour"]),
+                                          dev(a["entropy"]), prio_cfg_of(w), None, q)
+    qh = q.cpu().numpy().view(np.uint32)
+    s, tq, ws = _build(qh)
+    u = np.random.default_rng(9).integers(0, 1 << 64, size=777, dtype=np.uint64)
+    idx, _ = _sample(s, u, w.beta)
+    np.testing.assert_array_equal(idx, sample_by_prefix(qh, u))
+    b = torch.full((777,), -7, dtype=torch.int64, device="cuda")
+    e = torch.full((777,), -7, dtype=torch.int64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    distrl.distrl_trajectory_ranges(dev(off), dev(idx), b, e, status=status)
+    torch.cuda.synchronize()
+    rb, re = oracle.trajectory_ranges(off, idx)
+    np.testing.assert_array_equal(b.cpu().numpy(), rb)
+    np.testing.assert_array_equal(e.cpu().numpy(), re)
+    assert status.item() == 0
+    bad = np.array([0, m, -1, m - 1], dtype=np.int64)
+    b2 = torch.zeros(4, dtype=torch.int64, device="cuda")
+    e2 = torch.zeros(4, dtype=torch.int64, device="cuda")
+    distrl.distrl_trajectory_ranges(dev(off), dev(bad), b2, e2, status=status)
+    torch.cuda.synchronize()
+    assert b2.cpu().tolist() == [int(off[0]), -1, -1, int(off[m - 1])]
+    assert e2.cpu().tolist() == [int(off[1]), -1, -1, int(off[m])]
+    assert status.item() != 0
+    s.close()
