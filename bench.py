@@ -397,7 +397,8 @@ def run_ours(args):
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     # ---- the entry points beyond the main path, each timed alone on the same buffer (not part of `value`):
-    # Monte-Carlo returns + labels, trajectory-level priorities, and a circular overwrite of 2^20 slots
+    # Monte-Carlo returns + labels, trajectory-level priorities, a circular overwrite of 2^20 slots, and the
+    # actor-loss coefficients of the whole buffer and of one drawn batch
     next_rows = None
     if args.next_rows and not tok:
         def timed(fn, reps=20):
@@ -422,11 +423,28 @@ def run_ours(args):
         new_q = torch.randint(1, 1 << 24, (k_over,), dtype=torch.int32, device="cuda")
         t_ov = timed(lambda: distrl.distrl_replay_overwrite(s_tmp, n - k_over // 2, new_q))
         s_tmp.close()
+        coef_all, coef_k = f32(), torch.empty(k, dtype=torch.float32, device="cuda")
+        t_ca = timed(lambda: distrl.distrl_actor_coefficients(ins.lp_buf, ins.lm_buf, adv, coef_all))
+        # one drawn batch: 20 calls (one per round's batch) replayed from a CUDA graph, so that the
+        # figure is the device's and not the Python caller's
+        def coef_batches():
+            for r in range(20):
+                distrl.distrl_actor_coefficients(ins.lp_buf, ins.lm_buf, adv, coef_k, idx=idx[r % R],
+                                                 is_weight=wts[r % R])
+        coef_batches()
+        torch.cuda.synchronize()
+        g_ck = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_ck):
+            coef_batches()
+        t_ck = timed(g_ck.replay) / 20
         mc_bytes, tr_bytes = 9 * n + 8 * (w.m + 1), 16 * n + 8 * (w.m + 1) + 4 * w.m
         next_rows = {
             "mc_returns": {"ms": t_mc * 1e3, "gbs": mc_bytes / t_mc / 1e9, "frac": mc_bytes / t_mc / 1e9 / _peaks()[0]},
             "priorities_traj": {"ms": t_tr * 1e3, "gbs": tr_bytes / t_tr / 1e9, "frac": tr_bytes / t_tr / 1e9 / _peaks()[0]},
             "replay_overwrite": {"slots": k_over, "ms": t_ov * 1e3, "slots_per_s": k_over / t_ov},
+            "actor_coefficients_buffer": {"ms": t_ca * 1e3, "gbs": 16 * n / t_ca / 1e9,
+                                          "frac": 16 * n / t_ca / 1e9 / _peaks()[0]},
+            "actor_coefficients_batch": {"k": k, "us": t_ck * 1e6},
         }
         if distrl.distrl_get_status(ws_r) or distrl.distrl_get_status(ws_s):
             raise SystemExit("device status after the extra entry points")

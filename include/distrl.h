@@ -282,7 +282,8 @@ int distrl_retrace_priorities_build(const distrl_batch *batch, float gamma, floa
  * enters with the scalar
  *   coef[j] = is_weight[j] * rho_i * A_i,   rho_i = exp(logp_target[i] - logp_behaviour[i]).
  *   idx       : [k] device indices into the buffer (e.g. from distrl_sample), or
- *               NULL with k == n for the whole buffer in order.
+ *               NULL with k == n for the whole buffer in order (k == 0: nothing
+ *               is done; any other k with idx NULL is DISTRL_ERR_SIZE).
  *   advantage : [n], e.g. the output of distrl_retrace_targets.
  *   is_weight : [k] importance-sampling weights from distrl_sample, or NULL (= 1).
  *   coef      : [k] output.

@@ -94,8 +94,8 @@ extern "C" int distrl_actor_coefficients(int64_t n, const int64_t *idx, int64_t 
                                          const float *is_weight, float *coef, int *status_out_device,
                                          void *stream) {
     if (n < 0 || n > DISTRL_MAX_N || k < 0 || k > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
-    if (!idx && k != n) return DISTRL_ERR_SIZE;
     if (k == 0) return DISTRL_OK;
+    if (!idx && k != n) return DISTRL_ERR_SIZE;
     if (!logp_target || !logp_behaviour || !advantage || !coef) return DISTRL_ERR_NULL;
     const void *ptrs[] = {logp_target, logp_behaviour, advantage, is_weight, coef, status_out_device};
     bool vec = true;
