@@ -41,18 +41,22 @@ __global__ void __launch_bounds__(kPrioThreads) priority_kernel(
 }
 
 // Trajectory means: a block takes kPrioThreads consecutive trajectories, whose steps are one
-// contiguous range of the buffer.  All threads stream that range with coalesced loads, a window of
-// kTrajWindow steps at a time, and leave the three per-step terms (|delta|, min(rho, clip), H) in
-// shared memory; then every thread adds up the part of its own trajectory that lies in the window.
-// The formula is applied to the means at the end.
+// contiguous range of the buffer.  All threads stream that range, a window of kTrajWindow steps at a
+// time (16-byte loads when the arrays are 16-byte aligned; windows then start on multiples of four
+// steps), and leave one number per step in shared memory; then every thread adds up the part of its
+// own trajectory that lies in the window.  The priority is linear in the three means, so the number
+// kept per step is the whole combination w_td |delta_t| + w_rho min(rho_t, clip) + w_ent H_t and its
+// trajectory mean is the priority: one sum per trajectory instead of three.
 constexpr int kTrajWindow = 2048;
 
+template <bool VEC>
 __global__ void __launch_bounds__(kPrioThreads) priority_traj_kernel(
     int64_t n, int64_t m, const int64_t *__restrict__ off, const float *__restrict__ delta,
     const float *__restrict__ lp, const float *__restrict__ lm, const float *__restrict__ ent, PrioCfg c,
     float *__restrict__ mass_out, uint32_t *__restrict__ q_out) {
-    __shared__ float s_d[kTrajWindow], s_r[kTrajWindow], s_h[kTrajWindow];
+    __shared__ __align__(16) float s_x[kTrajWindow];
     const int tid = threadIdx.x;
+    constexpr float kLog2e = 1.4426950408889634f;
     auto inside = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > n ? n : x); };
     const int64_t chunks = (m + kPrioThreads - 1) / kPrioThreads;
     for (int64_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) { // block-uniform
@@ -67,44 +71,81 @@ __global__ void __launch_bounds__(kPrioThreads) priority_traj_kernel(
         const int64_t A = inside(off[j0]);
         int64_t B = inside(off[j1]);
         if (B < A) B = A;
-        float sd = 0.f, sr = 0.f, sh = 0.f;
-        for (int64_t p = A; p < B; p += kTrajWindow) {
+        auto term = [&](float d, float x, float y, float h) { // h: the entropy, read only if given
+            const float rho = fminf(exp2f((x - y) * kLog2e), c.rho_clip);
+            return c.w_td * fabsf(d) + c.w_rho * rho + c.w_ent * (ent ? h : -x);
+        };
+        float sum = 0.f;
+        for (int64_t p = VEC ? (A & ~(int64_t)3) : A; p < B; p += kTrajWindow) {
             const int cnt = (int)((B - p < kTrajWindow) ? B - p : kTrajWindow);
-            for (int i0 = tid; i0 < cnt; i0 += 4 * kPrioThreads) { // 16 loads in flight per thread
-                float vd[4], vp[4], vm[4], ve[4];
+            if (VEC) {
+                // four consecutive steps per thread and load; a group that reaches past the buffer's
+                // end is fetched step by step.  Steps before A or at and after B belong to other
+                // blocks: whatever lands in their slots is never added up.
+                float4 vd[2], vp[2], vm[2], ve[2];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int i = i0 + u * kPrioThreads;
-                    const int64_t t = p + (i < cnt ? i : i0);
-                    vd[u] = __ldcs(delta + t);
-                    vp[u] = __ldcs(lp + t);
-                    vm[u] = __ldcs(lm + t);
-                    ve[u] = ent ? __ldcs(ent + t) : 0.f;
+                for (int u = 0; u < 2; ++u) {
+                    const int i = 4 * tid + u * 4 * kPrioThreads;
+                    const int64_t t = p + i;
+                    if (i < cnt && t + 4 <= n) {
+                        vd[u] = __ldcs(reinterpret_cast<const float4 *>(delta + t));
+                        vp[u] = __ldcs(reinterpret_cast<const float4 *>(lp + t));
+                        vm[u] = __ldcs(reinterpret_cast<const float4 *>(lm + t));
+                        ve[u] = ent ? __ldcs(reinterpret_cast<const float4 *>(ent + t)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    } else {
+                        float q[4][4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const bool ok = i < cnt && t + e < n;
+                            q[0][e] = ok ? delta[t + e] : 0.f;
+                            q[1][e] = ok ? lp[t + e] : 0.f;
+                            q[2][e] = ok ? lm[t + e] : 0.f;
+                            q[3][e] = (ok && ent) ? ent[t + e] : 0.f;
+                        }
+                        vd[u] = make_float4(q[0][0], q[0][1], q[0][2], q[0][3]);
+                        vp[u] = make_float4(q[1][0], q[1][1], q[1][2], q[1][3]);
+                        vm[u] = make_float4(q[2][0], q[2][1], q[2][2], q[2][3]);
+                        ve[u] = make_float4(q[3][0], q[3][1], q[3][2], q[3][3]);
+                    }
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int i = i0 + u * kPrioThreads;
-                    if (i < cnt) {
-                        s_d[i] = fabsf(vd[u]);
-                        s_r[i] = fminf(expf(vp[u] - vm[u]), c.rho_clip);
-                        s_h[i] = ent ? ve[u] : -vp[u];
+                for (int u = 0; u < 2; ++u) {
+                    const int i = 4 * tid + u * 4 * kPrioThreads;
+                    if (i < cnt)
+                        *reinterpret_cast<float4 *>(s_x + i) = make_float4(
+                            term(vd[u].x, vp[u].x, vm[u].x, ve[u].x), term(vd[u].y, vp[u].y, vm[u].y, ve[u].y),
+                            term(vd[u].z, vp[u].z, vm[u].z, ve[u].z), term(vd[u].w, vp[u].w, vm[u].w, ve[u].w));
+                }
+            } else {
+                for (int i0 = tid; i0 < cnt; i0 += 4 * kPrioThreads) { // 16 loads in flight per thread
+                    float vd[4], vp[4], vm[4], ve[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int i = i0 + u * kPrioThreads;
+                        const int64_t t = p + (i < cnt ? i : i0);
+                        vd[u] = __ldcs(delta + t);
+                        vp[u] = __ldcs(lp + t);
+                        vm[u] = __ldcs(lm + t);
+                        ve[u] = ent ? __ldcs(ent + t) : 0.f;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int i = i0 + u * kPrioThreads;
+                        if (i < cnt) s_x[i] = term(vd[u], vp[u], vm[u], ve[u]);
                     }
                 }
             }
             __syncthreads();
-            const int64_t lo = (a > p) ? a : p, hi = (b < p + cnt) ? b : p + cnt;
-            for (int64_t t = lo; t < hi; ++t) {
-                sd += s_d[t - p];
-                sr += s_r[t - p];
-                sh += s_h[t - p];
-            }
+            const int64_t lo64 = ((a > p) ? a : p) - p, hi64 = ((b < p + cnt) ? b : p + cnt) - p;
+            const int lo = (int)(lo64 < cnt ? lo64 : cnt), hi = (int)(hi64 > 0 ? hi64 : 0); // both in [0, cnt]
+            for (int t = lo; t < hi; ++t) sum += s_x[t];
             __syncthreads();
         }
         if (j < m) {
             float ms = 0.f;
             if (b > a) {
                 const float inv = 1.f / (float)(b - a);
-                const float pr = c.w_td * (sd * inv) + c.w_rho * (sr * inv) + c.w_ent * (sh * inv);
+                const float pr = sum * inv;
                 ms = (c.alpha == 0.5f) ? sqrtf(pr) : (c.alpha == 1.0f) ? pr : powf(pr, c.alpha);
             }
             if (mass_out) mass_out[j] = ms;
@@ -159,14 +200,23 @@ extern "C" int distrl_compute_priorities_traj(int64_t n, int64_t m, const int64_
     int rc = check_prio_cfg(cfg, &c);
     if (rc) return rc;
     if (m == 0) return DISTRL_OK;
-    if (!off || !td_delta || !lp || !lm || !prio_q) return DISTRL_ERR_NULL;
+    if (!off || !prio_q) return DISTRL_ERR_NULL;
+    if (n > 0 && (!td_delta || !lp || !lm)) return DISTRL_ERR_NULL; // n == 0: only empty trajectories, nothing is read
     const void *ptrs[] = {td_delta, lp, lm, entropy, prio_mass_out, prio_q};
     for (const void *p : ptrs)
         if (p && !aligned_to(p, 4)) return DISTRL_ERR_ALIGN;
     if (!aligned_to(off, 8)) return DISTRL_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    priority_traj_kernel<<<grid_for(m, kPrioThreads, 148 * 8), kPrioThreads, 0, st>>>(
-        n, m, off, td_delta, lp, lm, entropy, c, prio_mass_out, prio_q);
+    bool vec = true;
+    for (const void *p : {(const void *)td_delta, (const void *)lp, (const void *)lm, (const void *)entropy})
+        if (p && !aligned_to(p, 16)) vec = false;
+    const int grid = grid_for(m, kPrioThreads, 148 * 8);
+    if (vec)
+        priority_traj_kernel<true><<<grid, kPrioThreads, 0, st>>>(n, m, off, td_delta, lp, lm, entropy, c,
+                                                                  prio_mass_out, prio_q);
+    else
+        priority_traj_kernel<false><<<grid, kPrioThreads, 0, st>>>(n, m, off, td_delta, lp, lm, entropy, c,
+                                                                   prio_mass_out, prio_q);
     DISTRL_CUDA_TRY(cudaGetLastError());
     return DISTRL_OK;
 }

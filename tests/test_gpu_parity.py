@@ -294,6 +294,49 @@ def test_trajectory_level_priorities():
     np.testing.assert_array_equal(q.cpu().numpy().view(np.uint32), oracle.quantise(mass.cpu().numpy(), w.scale))
 
 
+def _traj_layouts():
+    rng = np.random.default_rng(77)
+    yield "ones", np.ones(3000, dtype=np.int64)
+    yield "rows_of_32", np.full(700, 32, dtype=np.int64)
+    yield "31_33", np.tile(np.array([31, 33], dtype=np.int64), 400)
+    yield "window_edges", np.array([2048, 2047, 1, 2049, 4096, 5, 6000, 255, 257, 256], dtype=np.int64)
+    yield "one_long", np.array([50_001], dtype=np.int64)
+    yield "empties_everywhere", np.concatenate([np.zeros(600, dtype=np.int64), [7], np.zeros(300, dtype=np.int64),
+                                                rng.integers(0, 4, 900), [3000], np.zeros(5, dtype=np.int64)])
+    yield "geometric_mix", np.minimum(rng.geometric(1 / 12.0, 5000), 200).astype(np.int64)
+    yield "long_and_short", np.where(rng.random(1500) < 0.02, rng.integers(500, 3000, 1500), rng.integers(1, 6, 1500))
+    yield "all_empty", np.zeros(300, dtype=np.int64)
+
+
+@pytest.mark.parametrize("name,lens", list(_traj_layouts()), ids=[nm for nm, _ in _traj_layouts()])
+@pytest.mark.parametrize("with_entropy", [True, False])
+def test_trajectory_level_priorities_layouts(name, lens, with_entropy):
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    n, m = int(off[-1]), lens.shape[0]
+    rng = np.random.default_rng(m + n)
+    delta = (rng.normal(0, 1, n) * np.exp(rng.normal(0, 1, n))).astype(np.float32)
+    lm = rng.normal(-5, 2, n).astype(np.float32)
+    lp = (lm + rng.normal(0, 0.7, n)).astype(np.float32)
+    ent = rng.uniform(0, 3, n).astype(np.float32)
+    w = synth.make_workload(0)
+    mass = torch.full((m,), float("nan"), dtype=torch.float32, device="cuda")
+    q = torch.zeros(m, dtype=torch.int32, device="cuda")
+    one = lambda x: dev(x) if n else torch.empty(0, dtype=torch.float32, device="cuda")
+    runs = []
+    for _ in range(3):
+        distrl.distrl_compute_priorities_traj(dev(off), one(delta), one(lp), one(lm), one(ent) if with_entropy else None,
+                                              prio_cfg_of(w), mass, q)
+        torch.cuda.synchronize()
+        runs.append((mass.cpu().numpy().copy(), q.cpu().numpy().copy()))
+    ref = oracle.priority_mass_traj(off, delta, lp, lm, ent if with_entropy else None, w.w_td, w.w_rho, w.w_ent,
+                                    w.rho_clip, w.alpha)
+    assert_close(runs[0][0], ref, "traj prio_mass (%s)" % name)
+    np.testing.assert_array_equal(runs[0][1].view(np.uint32), oracle.quantise(runs[0][0], w.scale))
+    for r in runs[1:]:                                   # every sum is formed in one fixed order
+        np.testing.assert_array_equal(r[0], runs[0][0])
+        np.testing.assert_array_equal(r[1], runs[0][1])
+
+
 # ------------------------------------------------------------------ sampler ---
 
 def _masses(n, seed, heavy=True):
