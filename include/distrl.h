@@ -177,8 +177,12 @@ int distrl_compute_priorities(int64_t n, const float *td_delta, const float *log
 
 /*
  * Trajectory-level priority exactly as Section 5.3 writes it: the same formula
- * applied to the trajectory means of |delta|, min(rho, rho_clip) and H.
+ * applied to the trajectory means of |delta|, min(rho, rho_clip) and H.  (The
+ * formula is linear in the means, so the kernel averages the per-step
+ * combination w_td|delta_t| + w_rho min(rho_t, rho_clip) + w_ent H_t: the same
+ * number up to fp32 rounding.)
  *   prio_mass : [M] or NULL;  prio_q : [M] required.  Empty trajectory: q = 1.
+ *   With n == 0 (only empty trajectories) the per-step arrays may be NULL.
  */
 int distrl_compute_priorities_traj(int64_t n, int64_t m, const int64_t *traj_offsets,
                                    const float *td_delta, const float *logp_target,
