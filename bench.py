@@ -485,7 +485,8 @@ def run_ours(args):
                      "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
                      "frac_of_nominal_8000": ach / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name) if (args.n_override is None and not args.fused) else None,
                      "algorithmic_bytes": retrace_bytes},
-        "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": METRIC, "ms_per_step": e2e_ms,
+        "e2e": {"value": world * n / (e2e_ms * 1e-3) if e2e_ms == e2e_ms else None, "unit": METRIC,
+                "ms_per_step": e2e_ms if e2e_ms == e2e_ms else None,   # None: leg skipped with --no-e2e
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clk,

@@ -91,3 +91,27 @@ def test_token_level_full_size_sampled_trajectories():
     assert_close(d_w.cpu().numpy(), oracle.is_weights(qh, want, w.beta, True), "is_weight")
     assert distrl.distrl_get_status(ws2) == 0
     s.close()
+
+
+def test_large_buffer_trajectory_priorities_and_actor_coefficients():
+    # workload 3 at its real size (16,777,216 steps, 1.4 M trajectories), every output against the oracle
+    from helpers import prio_cfg_of
+    w = synth.make_workload(3)
+    a = w.arrays
+    n, m, off = w.n, w.m, a["traj_offsets"]
+    rng = np.random.default_rng(11)
+    delta = (rng.standard_normal(n) * synth.heavy_tail_scale(w)).astype(np.float32)
+    adv = rng.standard_normal(n).astype(np.float32)
+    t_lp, t_lm, t_ent = dev(a["logp_target"]), dev(a["logp_behaviour"]), dev(a["entropy"])
+    mass = torch.empty(m, dtype=torch.float32, device="cuda")
+    q = torch.empty(m, dtype=torch.int32, device="cuda")
+    distrl.distrl_compute_priorities_traj(dev(off), dev(delta), t_lp, t_lm, t_ent, prio_cfg_of(w), mass, q)
+    coef = torch.empty(n, dtype=torch.float32, device="cuda")
+    distrl.distrl_actor_coefficients(t_lp, t_lm, dev(adv), coef)
+    torch.cuda.synchronize()
+    ref = oracle.priority_mass_traj(off, delta, a["logp_target"], a["logp_behaviour"], a["entropy"], w.w_td, w.w_rho,
+                                    w.w_ent, w.rho_clip, w.alpha)
+    assert_close(mass.cpu().numpy(), ref, "trajectory-level mass, full size")
+    np.testing.assert_array_equal(q.cpu().numpy().view(np.uint32), oracle.quantise(mass.cpu().numpy(), w.scale))
+    assert_close(coef.cpu().numpy(), oracle.actor_coefficients(a["logp_target"], a["logp_behaviour"], adv),
+                 "actor coefficients, full size", tol=1e-5)
