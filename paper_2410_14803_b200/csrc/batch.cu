@@ -78,10 +78,9 @@ __global__ void __launch_bounds__(kBatchThreads) traj_ranges_kernel(
     }
 }
 
-static int batch_grid(int64_t items) {
+static int batch_grid(int64_t items, int64_t cap) { // cap: one resident wave of the kernel
     int64_t b = ceil_div(items, kBatchThreads);
     if (b < 1) b = 1;
-    const int64_t cap = 148 * 8; // 148 SMs x 8 resident blocks of 256 threads
     return (int)(b > cap ? cap : b);
 }
 
@@ -105,15 +104,19 @@ extern "C" int distrl_actor_coefficients(int64_t n, const int64_t *idx, int64_t 
     }
     if (idx && !aligned_to(idx, 8)) return DISTRL_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (idx)
-        actor_gather_kernel<<<batch_grid(k), kBatchThreads, 0, st>>>(n, k, idx, logp_target, logp_behaviour,
-                                                                     advantage, is_weight, coef, status_out_device);
-    else if (vec)
-        actor_stream_kernel<true><<<batch_grid(n / 4 + 1), kBatchThreads, 0, st>>>(n, logp_target, logp_behaviour,
-                                                                                   advantage, is_weight, coef);
-    else
-        actor_stream_kernel<false><<<batch_grid(n), kBatchThreads, 0, st>>>(n, logp_target, logp_behaviour,
-                                                                            advantage, is_weight, coef);
+    if (idx) {
+        const int grid = batch_grid(k, one_wave_blocks(actor_gather_kernel, kBatchThreads));
+        actor_gather_kernel<<<grid, kBatchThreads, 0, st>>>(n, k, idx, logp_target, logp_behaviour, advantage,
+                                                            is_weight, coef, status_out_device);
+    } else if (vec) {
+        const int grid = batch_grid(n / 4 + 1, one_wave_blocks(actor_stream_kernel<true>, kBatchThreads));
+        actor_stream_kernel<true><<<grid, kBatchThreads, 0, st>>>(n, logp_target, logp_behaviour, advantage,
+                                                                  is_weight, coef);
+    } else {
+        const int grid = batch_grid(n, one_wave_blocks(actor_stream_kernel<false>, kBatchThreads));
+        actor_stream_kernel<false><<<grid, kBatchThreads, 0, st>>>(n, logp_target, logp_behaviour, advantage,
+                                                                   is_weight, coef);
+    }
     DISTRL_CUDA_TRY(cudaGetLastError());
     return DISTRL_OK;
 }
@@ -126,8 +129,9 @@ extern "C" int distrl_trajectory_ranges(int64_t m, const int64_t *traj_offsets, 
     if (!aligned_to(traj_offsets, 8) || !aligned_to(idx, 8) || !aligned_to(begin, 8) || !aligned_to(end, 8) ||
         (status_out_device && !aligned_to(status_out_device, 4)))
         return DISTRL_ERR_ALIGN;
-    traj_ranges_kernel<<<batch_grid(k), kBatchThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        m, traj_offsets, k, idx, begin, end, status_out_device);
+    const int grid = batch_grid(k, one_wave_blocks(traj_ranges_kernel, kBatchThreads));
+    traj_ranges_kernel<<<grid, kBatchThreads, 0, static_cast<cudaStream_t>(stream)>>>(m, traj_offsets, k, idx, begin,
+                                                                                     end, status_out_device);
     DISTRL_CUDA_TRY(cudaGetLastError());
     return DISTRL_OK;
 }

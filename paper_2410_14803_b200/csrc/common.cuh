@@ -46,6 +46,21 @@ static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 b
 }
 #endif
 
+// Blocks of one resident wave of `kernel` on the current device: a grid-stride kernel launched with
+// more blocks than fit at once ends with a partly filled second wave.
+#ifdef __CUDACC__
+template <typename K>
+static inline int one_wave_blocks(K kernel, int threads, size_t smem = 0) {
+    int dev = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem) != cudaSuccess || per_sm <= 0)
+        per_sm = 4;
+    return sms * per_sm;
+}
+#endif
+
 // Every workspace starts with this header (256 bytes reserved).
 struct WorkspaceHeader {
     int status;          // sticky device-side status word (distrl_status)

@@ -180,13 +180,13 @@ extern "C" int distrl_compute_priorities(int64_t n, const float *td_delta, const
         if (p && !aligned_to(p, 16)) vec = false;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // 148 SMs x 8 resident blocks of 256 threads
+    // one resident wave of blocks, each striding over the buffer
     if (vec)
-        priority_kernel<true><<<grid_for(n / 4 + 1, kPrioThreads, 148 * 8), kPrioThreads, 0, st>>>(
-            n, td_delta, lp, lm, entropy, c, prio_mass_out, prio_q);
+        priority_kernel<true><<<grid_for(n / 4 + 1, kPrioThreads, one_wave_blocks(priority_kernel<true>, kPrioThreads)),
+                                kPrioThreads, 0, st>>>(n, td_delta, lp, lm, entropy, c, prio_mass_out, prio_q);
     else
-        priority_kernel<false><<<grid_for(n, kPrioThreads, 148 * 8), kPrioThreads, 0, st>>>(
-            n, td_delta, lp, lm, entropy, c, prio_mass_out, prio_q);
+        priority_kernel<false><<<grid_for(n, kPrioThreads, one_wave_blocks(priority_kernel<false>, kPrioThreads)),
+                                 kPrioThreads, 0, st>>>(n, td_delta, lp, lm, entropy, c, prio_mass_out, prio_q);
     DISTRL_CUDA_TRY(cudaGetLastError());
     return DISTRL_OK;
 }
@@ -210,7 +210,9 @@ extern "C" int distrl_compute_priorities_traj(int64_t n, int64_t m, const int64_
     bool vec = true;
     for (const void *p : {(const void *)td_delta, (const void *)lp, (const void *)lm, (const void *)entropy})
         if (p && !aligned_to(p, 16)) vec = false;
-    const int grid = grid_for(m, kPrioThreads, 148 * 8);
+    // one wave: as many blocks as are resident at once, each striding over its share of the chunks
+    const int grid = grid_for(m, kPrioThreads, vec ? one_wave_blocks(priority_traj_kernel<true>, kPrioThreads)
+                                                   : one_wave_blocks(priority_traj_kernel<false>, kPrioThreads));
     if (vec)
         priority_traj_kernel<true><<<grid, kPrioThreads, 0, st>>>(n, m, off, td_delta, lp, lm, entropy, c,
                                                                   prio_mass_out, prio_q);
