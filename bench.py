@@ -474,12 +474,14 @@ def run_ours(args):
         "config": _config(w, args, l2="inputs larger than L2 (%.0f MB touched per step)" %
                           ((retrace_bytes + prio_bytes + build_bytes) / 1e6)),
         "stages": {
-            "retrace_ms": float(stage_ms[0]), "priorities_ms": float(stage_ms[1]), "build_sampler_ms": float(stage_ms[2]),
+            # with --fused the first stage is the one fused pass and the next two are empty
+            "retrace_ms": float(stage_ms[0]), "priorities_ms": None if args.fused else float(stage_ms[1]),
+            "build_sampler_ms": None if args.fused else float(stage_ms[2]),
             "rounds_ms": float(stage_ms[3]), "us_per_round": float(1e3 * stage_ms[3] / R),
             "retrace_priority_transitions_per_s": n / ((stage_ms[0] + stage_ms[1]) * 1e-3),
             "samples_per_s": R * k / (stage_ms[3] * 1e-3),
-            "priorities_gbs": prio_bytes / (stage_ms[1] * 1e-3) / 1e9,
-            "build_sampler_gbs": build_bytes / (stage_ms[2] * 1e-3) / 1e9,
+            "priorities_gbs": None if args.fused else prio_bytes / (stage_ms[1] * 1e-3) / 1e9,
+            "build_sampler_gbs": None if args.fused else build_bytes / (stage_ms[2] * 1e-3) / 1e9,
         },
         "roofline": {"bound": "hbm", "kernel": ("scan_mask_kernel + scan_pipe_kernel<fused> (distrl_retrace_priorities_build)" if args.fused else "scan_mask_kernel + %s (distrl_retrace_targets)" % ("scan_tok_pipe_kernel (+ two stand-ins that return at once)" if tok else "scan_pipe_kernel")), "achieved": ach, "peak": peak,
                      "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
