@@ -115,3 +115,29 @@ def test_large_buffer_trajectory_priorities_and_actor_coefficients():
     np.testing.assert_array_equal(q.cpu().numpy().view(np.uint32), oracle.quantise(mass.cpu().numpy(), w.scale))
     assert_close(coef.cpu().numpy(), oracle.actor_coefficients(a["logp_target"], a["logp_behaviour"], adv),
                  "actor coefficients, full size", tol=1e-5)
+
+
+def test_large_buffer_monte_carlo_returns():
+    # workload 3 at its real size: 8192 tiles, more than the persistent grid holds at once, so blocks take
+    # tiles by block number first and by ticket afterwards; every return and label against the oracle
+    w = synth.make_workload(3)
+    a = w.arrays
+    n = w.n
+    t_off, t_r = dev(a["traj_offsets"]), dev(a["rewards"])          # the batch holds pointers only
+    batch = distrl.make_batch(t_off, t_r, None)
+    G = torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")
+    lab = torch.full((n,), 7, dtype=torch.uint8, device="cuda")
+    ws = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws)
+    runs = []
+    for _ in range(3):
+        distrl.distrl_mc_returns(batch, w.gamma, G, lab, workspace=ws)
+        assert distrl.distrl_get_status(ws) == 0
+        runs.append(G.cpu().numpy().copy())
+    Gr, labr = oracle.mc_return(a["traj_offsets"], a["rewards"], w.gamma)
+    assert_close(runs[0], Gr, "mc_return, full size")
+    np.testing.assert_array_equal(lab.cpu().numpy(), (runs[0] > 0).astype(np.uint8))
+    clear = np.abs(Gr) > 1e-5
+    np.testing.assert_array_equal(lab.cpu().numpy()[clear], labr[clear])
+    for r in runs[1:]:
+        np.testing.assert_array_equal(r, runs[0])
