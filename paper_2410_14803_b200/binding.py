@@ -131,8 +131,11 @@ def make_prio_cfg(w_td=1.0, w_rho=0.5, w_ent=0.1, rho_clip=2.0, alpha=0.5, scale
 
 def make_batch(traj_offsets, rewards, values, logp_target=None, logp_behaviour=None, bootstrap_values=None,
                step_token_offsets=None, tok_logp_target=None, tok_logp_behaviour=None) -> distrl_batch:
-    """Fill a distrl_batch from CUDA tensors (kept alive by the caller)."""
+    """Fill a distrl_batch from CUDA tensors.  The struct holds device pointers only; the returned
+    object also keeps references to the tensors, so they live as long as it does."""
     b = distrl_batch()
+    b._tensors = (traj_offsets, rewards, values, logp_target, logp_behaviour, bootstrap_values,
+                  step_token_offsets, tok_logp_target, tok_logp_behaviour)
     b.struct_size = ctypes.sizeof(distrl_batch)
     b.n_transitions = rewards.numel()
     b.n_trajectories = traj_offsets.numel() - 1
