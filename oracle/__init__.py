@@ -229,3 +229,14 @@ def trajectory_ranges(traj_offsets, idx):
     if rc:
         raise IndexError("trajectory index outside [0, m)")
     return b, e
+
+
+def filter_trajectories(traj_offsets, traj_score, threshold, q):
+    """Zero, in place, the masses of every transition of trajectories scored below the threshold
+    (the V_traj filter of Section 5.1); returns how many trajectories are retained."""
+    assert q.dtype == np.uint32 and q.flags.c_contiguous
+    off, sc = _i64(traj_offsets), _f64(traj_score)
+    lib = _load()
+    lib.oracle_filter_trajectories.restype = ctypes.c_int64
+    return int(lib.oracle_filter_trajectories(_n(q.shape[0]), _n(off.shape[0] - 1), _p(off), _p(sc),
+                                              _d(threshold), _p(q)))

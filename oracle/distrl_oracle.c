@@ -331,3 +331,20 @@ int oracle_trajectory_ranges(int64_t m, const int64_t *off, int64_t k, const int
     }
     return 0;
 }
+
+/* Trajectory filter (Section 5.1 "Trajectory-Level Value Estimation", App. A "The trajectory value
+ * estimation function"): V_traj scores whole trajectories and the replay buffer retains only the
+ * high-value ones.  A trajectory is retained iff score >= threshold; every transition of a
+ * trajectory that is not retained gets sampling mass 0, so no proportional draw can return it.
+ * Returns the number of retained trajectories. */
+int64_t oracle_filter_trajectories(int64_t n, int64_t m, const int64_t *off, const double *score,
+                                   double threshold, uint32_t *q)
+{
+    (void)n;
+    int64_t kept = 0;
+    for (int64_t j = 0; j < m; ++j) {
+        if (score[j] >= threshold) { ++kept; continue; }
+        for (int64_t t = off[j]; t < off[j + 1]; ++t) q[t] = 0u;
+    }
+    return kept;
+}

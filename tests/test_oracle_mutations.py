@@ -57,6 +57,10 @@ MUTATIONS = {
         ("coef[j] = (w ? w[j] : 1.0) * rho * adv[i];", "coef[j] = rho * adv[i];"),
     "actor coefficient: advantage read at the batch position instead of the drawn index":
         ("coef[j] = (w ? w[j] : 1.0) * rho * adv[i];", "coef[j] = (w ? w[j] : 1.0) * rho * adv[j];"),
+    "filter keeps the low-scored trajectories instead of the high-scored ones":
+        ("if (score[j] >= threshold) { ++kept; continue; }", "if (score[j] < threshold) { ++kept; continue; }"),
+    "filter leaves a dropped trajectory's last transition in place":
+        ("for (int64_t t = off[j]; t < off[j + 1]; ++t) q[t] = 0u;", "for (int64_t t = off[j]; t < off[j + 1] - 1; ++t) q[t] = 0u;"),
     "trajectory range ends at its own start offset":
         ("end[j] = off[idx[j] + 1];", "end[j] = off[idx[j]];"),
 }

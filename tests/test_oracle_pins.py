@@ -416,3 +416,43 @@ def test_trajectory_ranges_tile_the_buffer():
         assert (pb[j], pe[j]) == (off[t], off[t + 1])
     with pytest.raises(IndexError):
         oracle.trajectory_ranges(off, [40])
+
+
+# ------------------------------------------------------- trajectory filter ---
+def test_filter_keeps_exactly_the_trajectories_at_or_above_the_threshold():
+    rng = np.random.default_rng(12)
+    lens = rng.integers(0, 7, 60)
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    n = int(off[-1])
+    q0 = rng.integers(1, 1000, n, dtype=np.uint64).astype(np.uint32)
+    score = rng.uniform(0, 1, 60)
+    score[3] = 0.5                 # exactly at the threshold: retained
+    score[4] = np.nan              # not comparable: not retained
+    q = q0.copy()
+    kept = oracle.filter_trajectories(off, score, 0.5, q)
+    assert kept == int(np.sum(score >= 0.5))
+    for j in range(60):            # independent restatement, trajectory by trajectory
+        seg = slice(int(off[j]), int(off[j + 1]))
+        if score[j] >= 0.5:
+            np.testing.assert_array_equal(q[seg], q0[seg])
+        else:
+            assert not q[seg].any()
+    # threshold below every score keeps all and changes nothing; above every score leaves nothing
+    q = q0.copy()
+    assert oracle.filter_trajectories(off, np.nan_to_num(score, nan=0.2), -1.0, q) == 60
+    np.testing.assert_array_equal(q, q0)
+    q = q0.copy()
+    assert oracle.filter_trajectories(off, score, 2.0, q) == 0 and not q.any()
+
+
+def test_no_draw_returns_a_filtered_transition_and_the_rest_keep_their_proportions():
+    off = np.array([0, 2, 2, 5, 6, 9], dtype=np.int64)            # five trajectories, one empty
+    q = np.array([3, 1, 4, 1, 5, 9, 2, 6, 5], dtype=np.uint32)
+    score = np.array([0.9, 0.9, 0.1, 0.7, 0.2])
+    assert oracle.filter_trajectories(off, score, 0.5, q) == 3
+    np.testing.assert_array_equal(q, [3, 1, 0, 0, 0, 9, 0, 0, 0])
+    total = int(q.sum())
+    # every threshold y in [0, total) by brute force: index i is hit exactly q_i times
+    u = np.array([((y << 64) + total - 1) // total for y in range(total)], dtype=np.uint64)
+    hits = np.bincount(oracle.sample_linear(q, u), minlength=9)
+    np.testing.assert_array_equal(hits, q)
