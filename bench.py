@@ -437,6 +437,9 @@ def run_ours(args):
         with torch.cuda.graph(g_ck):
             coef_batches()
         t_ck = timed(g_ck.replay) / 20
+        q_f = q.clone()
+        v_traj = torch.rand(w.m, dtype=torch.float32, device="cuda")       # stands in for V_traj's scores
+        t_fl = timed(lambda: distrl.distrl_filter_trajectories(ins.dv["traj_offsets"], v_traj, 0.5, q_f))
         mc_bytes, tr_bytes = 9 * n + 8 * (w.m + 1), 16 * n + 8 * (w.m + 1) + 4 * w.m
         next_rows = {
             "mc_returns": {"ms": t_mc * 1e3, "gbs": mc_bytes / t_mc / 1e9, "frac": mc_bytes / t_mc / 1e9 / _peaks()[0]},
@@ -445,6 +448,7 @@ def run_ours(args):
             "actor_coefficients_buffer": {"ms": t_ca * 1e3, "gbs": 16 * n / t_ca / 1e9,
                                           "frac": 16 * n / t_ca / 1e9 / _peaks()[0]},
             "actor_coefficients_batch": {"k": k, "us": t_ck * 1e6},
+            "filter_trajectories": {"ms": t_fl * 1e3, "dropped_fraction": 0.5, "transitions_per_s": n / t_fl},
         }
         if distrl.distrl_get_status(ws_r) or distrl.distrl_get_status(ws_s):
             raise SystemExit("device status after the extra entry points")

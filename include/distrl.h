@@ -312,6 +312,23 @@ int distrl_actor_coefficients(int64_t n, const int64_t *idx, int64_t k, const fl
 int distrl_trajectory_ranges(int64_t m, const int64_t *traj_offsets, const int64_t *idx, int64_t k,
                              int64_t *begin, int64_t *end, int *status_out_device, void *stream);
 
+/*
+ * Trajectory filter (Section 5.1 "Trajectory-Level Value Estimation"; App. A on
+ * V_traj: the estimator scores whole trajectories and the replay buffer retains
+ * only the high-value ones).  A trajectory is retained iff
+ * traj_score[j] >= threshold (a NaN score is not retained).  Every transition of
+ * a trajectory that is not retained gets prio_q = 0, so that no draw returns it;
+ * the transitions stay where they are until overwritten.  Masses of retained
+ * trajectories are left as they are.  Call it between distrl_compute_priorities
+ * and distrl_build_sampler (or rebuild the sampler afterwards); at least one
+ * retained trajectory must have a transition, or there is nothing to draw.
+ *   traj_score : [M] device scores (e.g. V_traj's outputs);  prio_q : [N] in/out.
+ *   kept_out_device : device uint64 or NULL; receives the number retained.
+ */
+int distrl_filter_trajectories(int64_t n, int64_t m, const int64_t *traj_offsets,
+                               const float *traj_score, float threshold, uint32_t *prio_q,
+                               uint64_t *kept_out_device, void *stream);
+
 /* Writes total = sum_i q_i to *total_out_device (a device uint64). */
 int distrl_sampler_total(distrl_sampler *s, uint64_t *total_out_device, void *stream);
 

@@ -84,6 +84,7 @@ def _load():
         "distrl_replay_overwrite": (ci, [vp, i64, i64, vp, vp]),
         "distrl_actor_coefficients": (ci, [i64, vp, i64, vp, vp, vp, vp, vp, vp, vp]),
         "distrl_trajectory_ranges": (ci, [i64, vp, vp, i64, vp, vp, vp, vp]),
+        "distrl_filter_trajectories": (ci, [i64, i64, vp, vp, f32, vp, vp, vp]),
         "distrl_sampler_total": (ci, [vp, vp, vp]),
         "distrl_sampler_level": (ci, [vp, ci, ctypes.POINTER(sz), ctypes.POINTER(i64)]),
         "distrl_destroy_sampler": (ci, [vp]),
@@ -324,6 +325,20 @@ def distrl_trajectory_ranges(traj_offsets: torch.Tensor, idx: torch.Tensor, begi
                                             _ptr(idx, torch.int64), k, _ptr(begin, torch.int64),
                                             _ptr(end, torch.int64), _ptr(status, torch.int32), _stream(stream)),
            "distrl_trajectory_ranges")
+
+
+def distrl_filter_trajectories(traj_offsets: torch.Tensor, traj_score: torch.Tensor, threshold: float,
+                               prio_q: torch.Tensor, kept_out: Optional[torch.Tensor] = None, stream=None):
+    """Zero the masses of every transition of trajectories scored below the threshold."""
+    m = traj_offsets.numel() - 1
+    if traj_score.numel() != m:
+        raise ValueError("one score per trajectory")
+    if prio_q.element_size() != 4:
+        raise ValueError("prio_q must hold 32-bit masses")
+    _check(_load().distrl_filter_trajectories(prio_q.numel(), m, _ptr(traj_offsets, torch.int64),
+                                              _ptr(traj_score, torch.float32), threshold, _ptr(prio_q),
+                                              _ptr(kept_out, torch.int64), _stream(stream)),
+           "distrl_filter_trajectories")
 
 
 def distrl_sampler_total(s: Sampler, total_out: torch.Tensor, stream=None):

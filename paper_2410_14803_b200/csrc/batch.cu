@@ -78,6 +78,43 @@ __global__ void __launch_bounds__(kBatchThreads) traj_ranges_kernel(
     }
 }
 
+// Trajectory filter: a block takes kBatchThreads consecutive trajectories, whose steps are one
+// contiguous range of the buffer, keeps their offsets and verdicts in shared memory, and sweeps the
+// range with coalesced accesses; a step finds its trajectory by binary search over the block's
+// offsets (among equal offsets the last one, i.e. the trajectory that is not empty) and writes a zero
+// mass if that trajectory is not retained.  Masses of retained trajectories are neither read nor
+// written.
+__global__ void __launch_bounds__(kBatchThreads) filter_kernel(
+    int64_t n, int64_t m, const int64_t *__restrict__ off, const float *__restrict__ score, float threshold,
+    uint32_t *__restrict__ q, unsigned long long *kept) {
+    __shared__ int64_t s_off[kBatchThreads + 1];
+    __shared__ unsigned char s_keep[kBatchThreads];
+    const int tid = threadIdx.x;
+    auto inside = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > n ? n : x); };
+    const int64_t chunks = (m + kBatchThreads - 1) / kBatchThreads;
+    for (int64_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) { // block-uniform
+        const int64_t j0 = chunk * kBatchThreads, j = j0 + tid;
+        const int nt = (int)((j0 + kBatchThreads < m) ? kBatchThreads : m - j0); // trajectories of this block
+        const bool keep = j < m && score[j] >= threshold;                        // NaN: not retained
+        if (tid <= nt) s_off[tid] = inside(off[j0 + tid]);
+        if (tid == 0 && nt == kBatchThreads) s_off[nt] = inside(off[j0 + nt]);
+        s_keep[tid] = keep ? 1 : 0;
+        const int kept_here = __syncthreads_count(keep);
+        if (tid == 0 && kept && kept_here) atomicAdd(kept, (unsigned long long)kept_here);
+        const int64_t A = s_off[0], B = s_off[nt];
+        for (int64_t t = A + tid; t < B; t += kBatchThreads) {
+            int lo = 0, hi = nt; // invariant: s_off[lo] <= t, and s_off[hi] > t or hi == nt
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (s_off[mid] <= t) lo = mid;
+                else hi = mid;
+            }
+            if (!s_keep[lo]) q[t] = 0u;
+        }
+        __syncthreads(); // the tables are reused by the next chunk
+    }
+}
+
 static int batch_grid(int64_t items, int64_t cap) { // cap: one resident wave of the kernel
     int64_t b = ceil_div(items, kBatchThreads);
     if (b < 1) b = 1;
@@ -132,6 +169,26 @@ extern "C" int distrl_trajectory_ranges(int64_t m, const int64_t *traj_offsets, 
     const int grid = batch_grid(k, one_wave_blocks(traj_ranges_kernel, kBatchThreads));
     traj_ranges_kernel<<<grid, kBatchThreads, 0, static_cast<cudaStream_t>(stream)>>>(m, traj_offsets, k, idx, begin,
                                                                                      end, status_out_device);
+    DISTRL_CUDA_TRY(cudaGetLastError());
+    return DISTRL_OK;
+}
+
+extern "C" int distrl_filter_trajectories(int64_t n, int64_t m, const int64_t *traj_offsets, const float *traj_score,
+                                          float threshold, uint32_t *prio_q, uint64_t *kept_out_device,
+                                          void *stream) {
+    if (n < 0 || m < 0 || n > DISTRL_MAX_N || m > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
+    if (!(threshold == threshold)) return DISTRL_ERR_PARAM;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (kept_out_device) {
+        if (!aligned_to(kept_out_device, 8)) return DISTRL_ERR_ALIGN;
+        DISTRL_CUDA_TRY(cudaMemsetAsync(kept_out_device, 0, sizeof(uint64_t), st));
+    }
+    if (m == 0) return DISTRL_OK;
+    if (!traj_offsets || !traj_score || (n > 0 && !prio_q)) return DISTRL_ERR_NULL;
+    if (!aligned_to(traj_offsets, 8) || !aligned_to(traj_score, 4) || !aligned_to(prio_q, 4)) return DISTRL_ERR_ALIGN;
+    const int grid = batch_grid(m, one_wave_blocks(filter_kernel, kBatchThreads));
+    filter_kernel<<<grid, kBatchThreads, 0, st>>>(n, m, traj_offsets, traj_score, threshold, prio_q,
+                                                  reinterpret_cast<unsigned long long *>(kept_out_device));
     DISTRL_CUDA_TRY(cudaGetLastError());
     return DISTRL_OK;
 }

@@ -1013,3 +1013,72 @@ def test_trajectory_level_draw_returns_transition_ranges():
     assert e2.cpu().tolist() == [int(off[1]), -1, -1, int(off[m])]
     assert status.item() != 0
     s.close()
+
+
+# ------------------------------------------------------------ trajectory filter ---
+
+@pytest.mark.parametrize("name,lens", list(_traj_layouts()), ids=[nm for nm, _ in _traj_layouts()])
+def test_filter_trajectories_layouts(name, lens):
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    n, m = int(off[-1]), lens.shape[0]
+    rng = np.random.default_rng(n + 3 * m)
+    q = rng.integers(1, 1 << 32, size=n, dtype=np.uint64).astype(np.uint32)
+    score = rng.uniform(0, 1, m).astype(np.float32)
+    score[rng.random(m) < 0.05] = np.float32(0.5)          # exactly at the threshold: retained
+    score[rng.random(m) < 0.02] = np.nan                   # not retained
+    tq = dev(q.view(np.int32)) if n else torch.empty(0, dtype=torch.int32, device="cuda")
+    kept = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+    distrl.distrl_filter_trajectories(dev(off), dev(score), 0.5, tq, kept)
+    torch.cuda.synchronize()
+    ref = q.copy()
+    kept_ref = oracle.filter_trajectories(off, score, 0.5, ref)
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), ref)
+    assert kept.item() == kept_ref
+
+
+def test_no_draw_returns_a_filtered_transition():
+    w = synth.make_workload(2)
+    a = w.arrays
+    off, n, m = a["traj_offsets"], w.n, w.m
+    g = gpu_retrace(off, a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"], w.gamma, w.lam)
+    _, q = _gpu_priorities(w, g["td_delta"])
+    score = np.random.default_rng(21).uniform(0, 1, m).astype(np.float32)   # stands in for V_traj's outputs
+    tq = dev(q.view(np.int32))
+    distrl.distrl_filter_trajectories(dev(off), dev(score), 0.6, tq)
+    ref = q.copy()
+    oracle.filter_trajectories(off, score, 0.6, ref)
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), ref)
+    ws = distrl.alloc_workspace(distrl.distrl_sampler_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws)
+    s = distrl.distrl_build_sampler(tq, ws)
+    _check_tree(s, ref)
+    u = np.random.default_rng(22).integers(0, 1 << 64, size=20000, dtype=np.uint64)
+    u[:3] = [0, (1 << 64) - 1, 1 << 63]
+    idx, wts = _sample(s, u, w.beta)
+    np.testing.assert_array_equal(idx, sample_by_prefix(ref, u))
+    traj_of = np.searchsorted(off, idx, side="right") - 1
+    assert np.all(score[traj_of] >= 0.6) and np.all(ref[idx] > 0)
+    assert_close(wts, oracle.is_weights(ref, idx, w.beta), "IS weights after filtering")
+    assert distrl.distrl_get_status(ws) == 0
+    s.close()
+
+
+def test_filter_trajectories_edges():
+    from paper_2410_14803_b200 import binding
+    off = np.array([0, 3, 3, 8], dtype=np.int64)
+    q = np.arange(1, 9, dtype=np.uint32)
+    tq = dev(q.view(np.int32))
+    kept = torch.zeros(1, dtype=torch.int64, device="cuda")
+    distrl.distrl_filter_trajectories(dev(off), dev(np.array([1, 1, 1], dtype=np.float32)), 0.0, tq, kept)   # all retained
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), q)
+    assert kept.item() == 3
+    distrl.distrl_filter_trajectories(dev(off), dev(np.array([0, 5, 5], dtype=np.float32)), 1.0, tq, kept)   # first dropped
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), [0, 0, 0, 4, 5, 6, 7, 8])
+    assert kept.item() == 2
+    with pytest.raises(distrl.DistrlError):
+        distrl.distrl_filter_trajectories(dev(off), dev(np.zeros(3, dtype=np.float32)), float("nan"), tq)
+    lib = binding._load()
+    assert lib.distrl_filter_trajectories(8, 0, None, None, 0.5, None, None, None) == binding.OK            # no trajectories
+    assert lib.distrl_filter_trajectories(8, 3, None, None, 0.5, tq.data_ptr(), None, None) == binding.ERR_NULL
