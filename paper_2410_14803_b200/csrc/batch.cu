@@ -79,39 +79,55 @@ __global__ void __launch_bounds__(kBatchThreads) traj_ranges_kernel(
 }
 
 // Trajectory filter: a block takes kBatchThreads consecutive trajectories, whose steps are one
-// contiguous range of the buffer, keeps their offsets and verdicts in shared memory, and sweeps the
-// range with coalesced accesses; a step finds its trajectory by binary search over the block's
-// offsets (among equal offsets the last one, i.e. the trajectory that is not empty) and writes a zero
-// mass if that trajectory is not retained.  Masses of retained trajectories are neither read nor
-// written.
+// contiguous range of the buffer, and walks that range in windows of kFilterWindow steps.  Per
+// window the thread of every trajectory that is not retained sets the bits of its steps in a
+// shared-memory bitmap (whole words at a time), then all threads sweep the window with coalesced
+// stores of zero where a bit is set.  Masses of retained trajectories are neither read nor written.
+constexpr int kFilterWindow = 4096;
+constexpr int kFilterWords = kFilterWindow / 32;
+
 __global__ void __launch_bounds__(kBatchThreads) filter_kernel(
     int64_t n, int64_t m, const int64_t *__restrict__ off, const float *__restrict__ score, float threshold,
     uint32_t *__restrict__ q, unsigned long long *kept) {
-    __shared__ int64_t s_off[kBatchThreads + 1];
-    __shared__ unsigned char s_keep[kBatchThreads];
+    __shared__ unsigned int s_drop[kFilterWords];
     const int tid = threadIdx.x;
     auto inside = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > n ? n : x); };
     const int64_t chunks = (m + kBatchThreads - 1) / kBatchThreads;
     for (int64_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) { // block-uniform
         const int64_t j0 = chunk * kBatchThreads, j = j0 + tid;
-        const int nt = (int)((j0 + kBatchThreads < m) ? kBatchThreads : m - j0); // trajectories of this block
-        const bool keep = j < m && score[j] >= threshold;                        // NaN: not retained
-        if (tid <= nt) s_off[tid] = inside(off[j0 + tid]);
-        if (tid == 0 && nt == kBatchThreads) s_off[nt] = inside(off[j0 + nt]);
-        s_keep[tid] = keep ? 1 : 0;
+        const int64_t j1 = (j0 + kBatchThreads < m) ? j0 + kBatchThreads : m;
+        int64_t a = 0, b = 0;
+        bool keep = false;
+        if (j < m) {
+            a = inside(off[j]);
+            b = inside(off[j + 1]);
+            if (b < a) b = a;
+            keep = score[j] >= threshold; // NaN: not retained
+        }
+        const int64_t A = inside(off[j0]);
+        int64_t B = inside(off[j1]);
+        if (B < A) B = A;
         const int kept_here = __syncthreads_count(keep);
         if (tid == 0 && kept && kept_here) atomicAdd(kept, (unsigned long long)kept_here);
-        const int64_t A = s_off[0], B = s_off[nt];
-        for (int64_t t = A + tid; t < B; t += kBatchThreads) {
-            int lo = 0, hi = nt; // invariant: s_off[lo] <= t, and s_off[hi] > t or hi == nt
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (s_off[mid] <= t) lo = mid;
-                else hi = mid;
+        const bool drop = j < m && !keep && b > a;
+        for (int64_t p = A; p < B; p += kFilterWindow) {
+            const int cnt = (int)((B - p < kFilterWindow) ? B - p : kFilterWindow);
+            if (tid < kFilterWords) s_drop[tid] = 0u;
+            __syncthreads();
+            if (drop && b > p && a < p + cnt) {
+                const int lo = (int)((a > p ? a : p) - p), hi = (int)((b < p + cnt ? b : p + cnt) - p); // [lo, hi) in [0, cnt]
+                for (int wd = lo >> 5; wd <= (hi - 1) >> 5; ++wd) {
+                    const int first = (wd == (lo >> 5)) ? (lo & 31) : 0;
+                    const int last = (wd == ((hi - 1) >> 5)) ? ((hi - 1) & 31) : 31; // inclusive
+                    const unsigned int bits = (0xFFFFFFFFu >> (31 - last)) & (0xFFFFFFFFu << first);
+                    atomicOr(&s_drop[wd], bits);
+                }
             }
-            if (!s_keep[lo]) q[t] = 0u;
+            __syncthreads();
+            for (int i = tid; i < cnt; i += kBatchThreads)
+                if ((s_drop[i >> 5] >> (i & 31)) & 1u) q[p + i] = 0u;
+            __syncthreads(); // the bitmap is cleared for the next window
         }
-        __syncthreads(); // the tables are reused by the next chunk
     }
 }
 
