@@ -61,6 +61,33 @@ MUTATIONS = {
         ("if (score[j] >= threshold) { ++kept; continue; }", "if (score[j] < threshold) { ++kept; continue; }"),
     "filter leaves a dropped trajectory's last transition in place":
         ("for (int64_t t = off[j]; t < off[j + 1]; ++t) q[t] = 0u;", "for (int64_t t = off[j]; t < off[j + 1] - 1; ++t) q[t] = 0u;"),
+    "refresh drops the entropy term":
+        ("double p = w_td * fabs(new_abs_delta[j]) + w_rho * fmin(rho, rho_clip) + w_ent * H;",
+         "double p = w_td * fabs(new_abs_delta[j]) + w_rho * fmin(rho, rho_clip);"),
+    "refresh: ratio inverted":
+        ("double rho = exp(logp_pi[i] - logp_mu[i]);\n        double H", "double rho = exp(logp_mu[i] - logp_pi[i]);\n        double H"),
+    "refresh: ratio not clipped":
+        ("double p = w_td * fabs(new_abs_delta[j]) + w_rho * fmin(rho, rho_clip) + w_ent * H;",
+         "double p = w_td * fabs(new_abs_delta[j]) + w_rho * rho + w_ent * H;"),
+    "refresh: entropy fallback has the wrong sign":
+        ("double H = entropy ? entropy[i] : -logp_pi[i];", "double H = entropy ? entropy[i] : logp_pi[i];"),
+    "refresh: entropy read at the batch position instead of the refreshed index":
+        ("double H = entropy ? entropy[i] : -logp_pi[i];", "double H = entropy ? entropy[j] : -logp_pi[i];"),
+    "refresh: exponent alpha ignored":
+        ("double mass = pow(p, alpha);\n        float mf", "double mass = p;\n        float mf"),
+    "trajectory priority: entropy fallback has the wrong sign":
+        ("sh += entropy ? entropy[t] : -logp_pi[t];", "sh += entropy ? entropy[t] : logp_pi[t];"),
+    "trajectory priority: ratio not clipped":
+        ("sr += fmin(exp(logp_pi[t] - logp_mu[t]), rho_clip);", "sr += exp(logp_pi[t] - logp_mu[t]);"),
+    "trajectory priority: ratio inverted":
+        ("sr += fmin(exp(logp_pi[t] - logp_mu[t]), rho_clip);", "sr += fmin(exp(logp_mu[t] - logp_pi[t]), rho_clip);"),
+    "trajectory priority: sums instead of means":
+        ("double p = w_td * (sd / (double)len) + w_rho * (sr / (double)len)", "double p = w_td * sd + w_rho * (sr / (double)len)"),
+    "priority: entropy fallback has the wrong sign":
+        ("double H = entropy ? entropy[t] : -logp_pi[t];", "double H = entropy ? entropy[t] : logp_pi[t];"),
+    "priority: ratio not clipped":
+        ("double p = w_td * fabs(td_delta[t]) + w_rho * fmin(rho, rho_clip) + w_ent * H;",
+         "double p = w_td * fabs(td_delta[t]) + w_rho * rho + w_ent * H;"),
     "trajectory range ends at its own start offset":
         ("end[j] = off[idx[j] + 1];", "end[j] = off[idx[j]];"),
 }

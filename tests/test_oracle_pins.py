@@ -333,6 +333,72 @@ def test_update_sequential_last_wins_and_equals_rebuild():
     assert tot == 5 * n + (3 << 20) - 5 + (2 << 20) - 5 + 1 - 5
 
 
+def test_update_priority_terms_by_hand():
+    # Every term of the Section 5.3 priority inside the refresh, worked by hand with alpha = 1:
+    #   p = w1 |delta_new| + w2 min(rho, clip) + w3 H,   w = (1, 0.5, 0.25), clip = 2
+    # index 1: rho = 1/2 (below the clip), H = 0.8  -> 3 + 0.25 + 0.2 = 3.45
+    # index 2: rho = 8   (clipped to 2),   H = 0.4  -> 1 + 1.0  + 0.1 = 2.1
+    # index 0: rho = 1,                    H = 2.0  -> 0 + 0.5  + 0.5 = 1.0   (delta sign is ignored below)
+    S = 2.0 ** 20
+    lp = np.array([0.0, math.log(0.25), math.log(0.5), -1.0])
+    lm = np.array([0.0, math.log(0.5), math.log(0.0625), -1.0])
+    ent = np.array([2.0, 0.8, 0.4, 9.0])
+    q = np.full(4, 7, dtype=np.uint32)
+    mass = oracle.update(q, [1, 2, 0], [3.0, -1.0, 0.0], lp, lm, ent, 1.0, 0.5, 0.25, 2.0, 1.0, S)
+    np.testing.assert_allclose(mass, [3.45, 2.1, 1.0], rtol=1e-15)
+    want = [1 << 20, int(np.rint(np.float64(np.float32(3.45)) * S)), int(np.rint(np.float64(np.float32(2.1)) * S)), 7]
+    assert q.tolist() == want
+    # alpha = 0.5 takes the square root of the same sums
+    q = np.full(4, 7, dtype=np.uint32)
+    mass = oracle.update(q, [1, 2, 0], [3.0, -1.0, 0.0], lp, lm, ent, 1.0, 0.5, 0.25, 2.0, 0.5, S)
+    np.testing.assert_allclose(mass, np.sqrt([3.45, 2.1, 1.0]), rtol=1e-15)
+    # no entropy array: H = -log pi(a|s) of the refreshed index.  Only that term: w = (0, 0, 1)
+    q = np.full(4, 7, dtype=np.uint32)
+    mass = oracle.update(q, [3, 1], [5.0, 5.0], lp, lm, None, 0.0, 0.0, 1.0, 2.0, 1.0, S)
+    np.testing.assert_allclose(mass, [1.0, math.log(4.0)], rtol=1e-15)
+    # only the ratio term, clip far away: the plain ratio pi / mu, not its inverse
+    q = np.full(4, 7, dtype=np.uint32)
+    mass = oracle.update(q, [1, 2], [5.0, 5.0], lp, lm, ent, 0.0, 1.0, 0.0, 100.0, 1.0, S)
+    np.testing.assert_allclose(mass, [0.5, 8.0], rtol=1e-15)
+
+
+def test_update_is_the_priority_of_the_fresh_delta_quantised():
+    # The refresh of index i with a fresh |delta| must leave exactly what the (separately pinned) priority and
+    # quantiser give for a buffer whose delta at i is the fresh one: update(q, idx, d_new) == Q(priority_mass(...))[idx].
+    rng = np.random.default_rng(21)
+    n, k, S = 300, 40, 2.0 ** 20
+    lm = rng.normal(-5, 2, n)
+    lp = lm + rng.normal(0, 1.0, n)           # ratios on both sides of the clip of 2
+    ent = rng.uniform(0, 3, n)
+    idx = rng.permutation(n)[:k]               # distinct, so the order does not matter here
+    d_new = np.abs(rng.normal(0, 1, k))
+    assert (np.exp(lp - lm)[idx] > 2.0).any() and (np.exp(lp - lm)[idx] < 2.0).any()
+    for entropy in (ent, None):
+        for alpha in (0.5, 1.0):
+            full = np.zeros(n)
+            full[idx] = d_new
+            ref_mass = oracle.priority_mass(full, lp, lm, entropy, 1.0, 0.5, 0.1, 2.0, alpha)
+            q = np.full(n, 3, dtype=np.uint32)
+            mass = oracle.update(q, idx, d_new, lp, lm, entropy, 1.0, 0.5, 0.1, 2.0, alpha, S)
+            np.testing.assert_array_equal(mass, ref_mass[idx])
+            want = np.full(n, 3, dtype=np.uint32)
+            want[idx] = oracle.quantise(ref_mass[idx].astype(np.float32), S)
+            np.testing.assert_array_equal(q, want)
+
+
+def test_trajectory_priority_without_entropy_uses_minus_log_pi():
+    # H_t = -log pi(a_t|s_t) averaged over the trajectory (Section 5.3), only that term switched on
+    lp = np.array([-1.0, -3.0, -0.5, -2.5, -4.0])
+    lm = lp.copy()
+    d = np.zeros(5)
+    out = oracle.priority_mass_traj([0, 2, 5], d, lp, lm, None, 0.0, 0.0, 1.0, 2.0, 1.0)
+    np.testing.assert_allclose(out, [2.0, 7.0 / 3.0], rtol=1e-15)
+    # and together with the other terms: w = (1, 0.5, 0.1), rho = 1 everywhere, |delta| mean 1.5 and 2
+    d = np.array([1.0, -2.0, 3.0, -1.0, 2.0])
+    out = oracle.priority_mass_traj([0, 2, 5], d, lp, lm, None, 1.0, 0.5, 0.1, 2.0, 1.0)
+    np.testing.assert_allclose(out, [1.5 + 0.5 + 0.2, 2.0 + 0.5 + 0.7 / 3.0], rtol=1e-15)
+
+
 def test_sampling_frequency_tracks_mass_after_update():
     # After an update the linear scan must see the new masses: enumerate again.
     q = np.array([2, 2, 2, 2], dtype=np.uint32)
