@@ -354,6 +354,18 @@ int distrl_get_status(void *workspace, void *stream);
  *   workspace : a retrace workspace (>= distrl_retrace_workspace_bytes(1024)). */
 int distrl_selftest_bounded_wait(void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * Library option (no counterpart in the paper).  A normalising distrl_sample whose
+ * grid fits the GPU lets its thread blocks wait for one another (batch maximum)
+ * and is therefore launched cooperatively: the driver puts the whole grid on the
+ * GPU at once, however busy other streams keep it.  With allowed = 0 (or when
+ * the driver refuses such a launch) the last block to finish normalises instead:
+ * correct under any scheduling, a little slower.  Process-wide; returns the old
+ * setting.  (The Retrace scan needs no such launch: its tiles go by ticket, so a
+ * block only ever waits for tiles of blocks that are already running.)
+ */
+int distrl_set_cooperative_launch(int allowed);
+
 const char *distrl_error_string(int code);
 const char *distrl_last_cuda_error(void); /* text of the last failed CUDA call, this thread */
 const char *distrl_version(void);

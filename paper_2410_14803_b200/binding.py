@@ -90,6 +90,7 @@ def _load():
         "distrl_destroy_sampler": (ci, [vp]),
         "distrl_get_status": (ci, [vp, vp]),
         "distrl_selftest_bounded_wait": (ci, [vp, sz, vp]),
+        "distrl_set_cooperative_launch": (ci, [ci]),
         "distrl_error_string": (ctypes.c_char_p, [ci]),
         "distrl_last_cuda_error": (ctypes.c_char_p, []),
         "distrl_version": (ctypes.c_char_p, []),
@@ -150,6 +151,11 @@ def make_batch(traj_offsets, rewards, values, logp_target=None, logp_behaviour=N
     b.tok_logp_target_bf16 = _ptr(tok_logp_target, torch.bfloat16)
     b.tok_logp_behaviour_bf16 = _ptr(tok_logp_behaviour, torch.bfloat16)
     return b
+
+
+def distrl_set_cooperative_launch(allowed: bool) -> bool:
+    """Library option: allow (default) or forbid the cooperative launch of a normalising draw; returns the old setting."""
+    return bool(_load().distrl_set_cooperative_launch(1 if allowed else 0))
 
 
 def distrl_version() -> str:

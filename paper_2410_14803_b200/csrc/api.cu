@@ -1,9 +1,13 @@
 // Library-wide entry points: status handling, error text, version.
 #include "common.cuh"
 
+#include <atomic>
 #include <cstdio>
 
 namespace distrl {
+
+static std::atomic<int> g_cooperative{1};
+bool cooperative_launch_allowed() { return g_cooperative.load(std::memory_order_relaxed) != 0; }
 
 static thread_local char g_cuda_error[256] = "";
 
@@ -51,6 +55,10 @@ extern "C" const char *distrl_error_string(int code) {
     case DISTRL_ERR_INDEX: return "index outside [0, n)";
     default: return "unknown status";
     }
+}
+
+extern "C" int distrl_set_cooperative_launch(int allowed) {
+    return g_cooperative.exchange(allowed ? 1 : 0, std::memory_order_relaxed);
 }
 
 extern "C" const char *distrl_last_cuda_error(void) { return g_cuda_error; }

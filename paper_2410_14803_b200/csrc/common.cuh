@@ -13,6 +13,10 @@ namespace distrl {
 // Records the text of a failed CUDA call for distrl_last_cuda_error().
 int record_cuda_error(cudaError_t e, const char *what);
 
+// Whether kernels whose blocks wait for one another may be launched cooperatively
+// (distrl_set_cooperative_launch; on by default).
+bool cooperative_launch_allowed();
+
 #define DISTRL_CUDA_TRY(expr)                                              \
     do {                                                                   \
         cudaError_t e__ = (expr);                                          \
@@ -70,7 +74,10 @@ struct WorkspaceHeader {
     unsigned int bad_epoch; // call number whose offsets failed validation (scan)
     unsigned int left;      // blocks that have taken the batch minimum and are leaving (sampler)
     unsigned int tok_dense; // token-level scan: the steps own too many tokens on average for the pipelined kernel
+    unsigned int pad_;
+    unsigned long long scan_ticket; // pipelined fp32 scan: (number of the call << 32) | tiles handed out so far
 };
+static_assert(sizeof(WorkspaceHeader) <= 256, "the header has 256 bytes");
 constexpr size_t kHeaderBytes = 256;
 
 // ---- device-side helpers ----------------------------------------------------

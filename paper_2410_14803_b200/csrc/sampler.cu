@@ -698,7 +698,7 @@ extern "C" int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k
         }
         fit = resident[dev];
     }
-    const int together = (normalise && is_weight_out && fit > 0 && blocks <= fit) ? 1 : 0;
+    const int together = (normalise && is_weight_out && fit > 0 && blocks <= fit && cooperative_launch_allowed()) ? 1 : 0;
     const unsigned long long *u64 = reinterpret_cast<const unsigned long long *>(u_fix);
     if (together) {
         // Blocks that wait for one another must all be on the GPU at the same time whatever else runs

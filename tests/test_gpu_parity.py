@@ -178,6 +178,60 @@ def test_retrace_repeated_runs_agree_bit_for_bit(kind):
     assert_close(first[2].view(np.float32), dl, "td_delta")
 
 
+def test_two_retrace_calls_at_the_same_time_on_two_streams():
+    # Trajectories far longer than the 128-step halo: almost every tile needs the value that its right
+    # neighbour produces, i.e. blocks wait for other blocks.  Two such calls on two streams (own
+    # workspaces) compete for the SMs; each must still finish with status 0 and the oracle's results,
+    # whichever way the device interleaves them (every tile goes by ticket, so a block only waits for
+    # tiles of blocks that are already running).
+    def case(seed, n, boot):
+        rng = np.random.default_rng(seed)
+        lens = []
+        while sum(lens) < n:
+            lens.append(int(rng.integers(300, 6000)))
+        lens[-1] -= sum(lens) - n
+        off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+        r, V, lp, lm = random_batch(seed, off)
+        lp = (lm + rng.normal(0, 0.05, n)).astype(np.float32)        # ratios near 1: the trace stays alive
+        b = rng.random(len(lens), dtype=np.float32) if boot else None
+        return off, r, V, lp, lm, b
+
+    cases = [case(41, 600_001, False), case(42, 450_000, False), case(43, 300_000, True)]
+    streams = [torch.cuda.Stream() for _ in cases]
+    held = []
+    for (off, r, V, lp, lm, b), st in zip(cases, streams):
+        n = r.shape[0]
+        t = dict(off=dev(off), r=dev(r), V=dev(V), lp=dev(lp), lm=dev(lm), b=dev(b) if b is not None else None)
+        t["batch"] = distrl.make_batch(t["off"], t["r"], t["V"], t["lp"], t["lm"], t["b"])
+        t["out"] = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(3)]
+        t["G"] = torch.empty(n, dtype=torch.float32, device="cuda")
+        t["ws"] = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+        t["ws2"] = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+        distrl.distrl_workspace_init(t["ws"])
+        distrl.distrl_workspace_init(t["ws2"])
+        held.append(t)
+    torch.cuda.synchronize()
+    for rnd in range(6):
+        for t in held:
+            for o in t["out"]:
+                o.fill_(float("nan"))
+            t["G"].fill_(float("nan"))
+        torch.cuda.synchronize()
+        for _ in range(3):           # several calls in flight on every stream
+            for t, st in zip(held, streams):
+                distrl.distrl_retrace_targets(t["batch"], 0.99, 0.95, *t["out"], workspace=t["ws"], stream=st)
+                distrl.distrl_mc_returns(t["batch"], 0.99, t["G"], None, workspace=t["ws2"], stream=st)
+        torch.cuda.synchronize()
+        for (off, r, V, lp, lm, b), t, st in zip(cases, held, streams):
+            assert distrl.distrl_get_status(t["ws"], stream=st) == 0
+            assert distrl.distrl_get_status(t["ws2"], stream=st) == 0
+            vt, adv, dl = oracle.retrace(off, r, V, lp, lm, 0.99, 0.95, bootstrap=b)
+            assert_close(t["out"][0].cpu().numpy(), vt, "v_target")
+            assert_close(t["out"][1].cpu().numpy(), adv, "advantage")
+            assert_close(t["out"][2].cpu().numpy(), dl, "td_delta")
+            assert_close(t["G"].cpu().numpy(), oracle.mc_return(off, r, 0.99)[0], "mc_return")
+
+
 def test_retrace_bad_offsets_are_reported_not_fatal():
     off = np.array([0, 10, 7, 20], dtype=np.int64)     # decreasing
     r, V, lp, lm = random_batch(1, np.array([0, 20]))
@@ -392,6 +446,27 @@ def test_sampler_build_and_sample(n, heavy):
     assert wts.max() == 1.0
     _, raw = _sample(s, u, 0.6, normalise=False)
     assert_close(raw, oracle.is_weights(q, idx, 0.6, False), "is_weight raw")
+    assert distrl.distrl_get_status(ws) == 0
+    s.close()
+
+
+def test_normalising_draw_without_a_cooperative_launch():
+    # the library option that forbids cooperative launches sends a normalising draw down the path of
+    # large batches (the last block rescales): same indices, same weights
+    q = _masses((1 << 20) + 3, 77)
+    s, tq, ws = _build(q)
+    u = np.random.default_rng(78).integers(0, 1 << 64, size=4096, dtype=np.uint64)
+    old = distrl.distrl_set_cooperative_launch(False)
+    try:
+        assert old is True
+        idx, wts = _sample(s, u, 0.4)
+    finally:
+        assert distrl.distrl_set_cooperative_launch(old) is False
+    idx2, wts2 = _sample(s, u, 0.4)
+    np.testing.assert_array_equal(idx, sample_by_prefix(q, u))
+    np.testing.assert_array_equal(idx, idx2)
+    assert_close(wts, oracle.is_weights(q, idx, 0.4, True), "is_weight")
+    assert_close(wts2, oracle.is_weights(q, idx, 0.4, True), "is_weight")
     assert distrl.distrl_get_status(ws) == 0
     s.close()
 
