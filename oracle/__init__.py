@@ -240,3 +240,43 @@ def filter_trajectories(traj_offsets, traj_score, threshold, q):
     lib.oracle_filter_trajectories.restype = ctypes.c_int64
     return int(lib.oracle_filter_trajectories(_n(q.shape[0]), _n(off.shape[0] - 1), _p(off), _p(sc),
                                               _d(threshold), _p(q)))
+
+
+class Ring:
+    """Circular replay buffer of whole trajectories (App. A "Circular Replay Buffer", Section 5.3): the
+    oracle's state.  ``fields`` are the per-transition fp64 arrays, ``q`` the masses, ``alive`` / ``start``
+    one flag per slot, ``head`` the next write index."""
+
+    def __init__(self, capacity: int, n_fields: int):
+        self.n = int(capacity)
+        self.fields = [np.zeros(self.n, dtype=np.float64) for _ in range(n_fields)]
+        self.q = np.zeros(self.n, dtype=np.uint32)
+        self.alive = np.zeros(self.n, dtype=np.uint8)
+        self.start = np.zeros(self.n, dtype=np.uint8)
+        self.start[0] = 1
+        self.head = 0
+
+    def ingest(self, new_offsets, new_fields, new_q) -> bool:
+        """Append trajectories (CSR offsets over the new rows); False if the call is refused."""
+        off = _i64(new_offsets)
+        k = off.shape[0] - 1
+        nf = [_f64(a) for a in new_fields]
+        assert len(nf) == len(self.fields)
+        nq = np.ascontiguousarray(new_q, dtype=np.uint32)
+        PP = ctypes.c_void_p * len(nf)
+        dst = PP(*[a.ctypes.data for a in self.fields])
+        src = PP(*[a.ctypes.data for a in nf])
+        head = ctypes.c_int64(self.head)
+        rc = _load().oracle_ring_ingest(_n(self.n), ctypes.c_int(len(nf)), dst, _p(self.q), _p(self.alive),
+                                        _p(self.start), ctypes.byref(head), _n(k), _p(off), src, _p(nq))
+        self.head = int(head.value)
+        return rc == 0
+
+    def segments(self):
+        """(offsets[M+1], alive[M]): the buffer as CSR segments, live trajectories and dead stretches."""
+        off = np.empty(self.n + 1, dtype=np.int64)
+        al = np.empty(self.n, dtype=np.uint8)
+        lib = _load()
+        lib.oracle_ring_segments.restype = ctypes.c_int64
+        m = int(lib.oracle_ring_segments(_n(self.n), _p(self.start), _p(self.alive), _p(off), _p(al)))
+        return off[:m + 1].copy(), al[:m].copy()

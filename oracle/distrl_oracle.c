@@ -348,3 +348,81 @@ int64_t oracle_filter_trajectories(int64_t n, int64_t m, const int64_t *off, con
     }
     return kept;
 }
+
+/* ------------------------------------------------------------------------- *
+ * Circular replay buffer of whole trajectories (App. A "Circular Replay Buffer": capacity N, the write
+ * index advances as i <- (i + 1) mod N, new experiences overwrite the oldest; Section 5.3 prioritises
+ * and replays trajectories).  Slots hold transitions; the flat buffer is cut into segments, each a
+ * live trajectory or a dead stretch:
+ *   start[i] = 1 : a segment starts at slot i (start[0] is always 1);
+ *   alive[i] = 1 : slot i belongs to a live trajectory;   q[i] : its sampling mass (0 when dead).
+ * A trajectory is stored in consecutive slots, because the Retrace recursion of Section 5.2 runs along
+ * it: one that would straddle the end of the buffer starts at slot 0 instead, and the slots left at the
+ * end are retired.  A stored trajectory that loses a slot is evicted as a whole: its remaining slots
+ * are dead, their masses 0, so no draw returns them.  New trajectories are taken in order; an empty one
+ * (length 0) stores nothing.  The call is refused (-1, nothing changed) if the offsets are not
+ * non-decreasing from 0, or if the write index would advance by more than N in this one call (rows
+ * plus retired slots), i.e. if the call would overwrite its own trajectories.
+ * ------------------------------------------------------------------------- */
+static void ring_kill_trajectory_at(int64_t n, uint32_t *q, uint8_t *alive, const uint8_t *start, int64_t i)
+{
+    if (!alive[i]) return;
+    int64_t s = i, e = i + 1;
+    while (!start[s]) --s;             /* first slot of the trajectory that owns slot i */
+    while (e < n && !start[e]) ++e;    /* one past its last slot */
+    for (int64_t t = s; t < e; ++t) { alive[t] = 0; q[t] = 0u; }
+}
+
+int oracle_ring_ingest(int64_t n, int n_fields, double *const *field, uint32_t *q, uint8_t *alive,
+                       uint8_t *start, int64_t *head, int64_t k, const int64_t *new_off,
+                       const double *const *new_field, const uint32_t *new_q)
+{
+    if (k < 0 || (k > 0 && new_off[0] != 0)) return -1;
+    {   /* dry run: how far would the write index travel? */
+        int64_t h = *head, advance = 0;
+        for (int64_t j = 0; j < k; ++j) {
+            int64_t T = new_off[j + 1] - new_off[j];
+            if (T < 0) return -1;
+            if (T == 0) continue;
+            if (h + T > n) { advance += n - h; h = 0; }
+            h += T;
+            advance += T;
+            if (advance > n) return -1;
+        }
+    }
+    int64_t h = *head;
+    for (int64_t j = 0; j < k; ++j) {
+        int64_t T = new_off[j + 1] - new_off[j];
+        if (T == 0) continue;
+        if (h + T > n) {               /* would straddle the end: retire [h, n), go on at slot 0 */
+            for (int64_t i = h; i < n; ++i) ring_kill_trajectory_at(n, q, alive, start, i);
+            for (int64_t i = h; i < n; ++i) start[i] = (i == h);
+            h = 0;
+        }
+        /* every stored trajectory that loses a slot goes as a whole */
+        for (int64_t i = h; i < h + T; ++i) ring_kill_trajectory_at(n, q, alive, start, i);
+        /* what follows the new trajectory starts a segment of its own */
+        if (h + T < n) start[h + T] = 1;
+        for (int64_t i = 0; i < T; ++i) {
+            for (int f = 0; f < n_fields; ++f) field[f][h + i] = new_field[f][new_off[j] + i];
+            q[h + i] = new_q[new_off[j] + i];
+            alive[h + i] = 1;
+            start[h + i] = (i == 0);
+        }
+        h += T;                        /* h == n wraps at the next write: (h + T) mod n */
+    }
+    *head = h % n;
+    return 0;
+}
+
+/* The segments as CSR offsets over the flat buffer, with one liveness flag per segment.
+ * Returns the number of segments M; off_out has M + 1 entries, the last one n. */
+int64_t oracle_ring_segments(int64_t n, const uint8_t *start, const uint8_t *alive, int64_t *off_out,
+                             uint8_t *seg_alive_out)
+{
+    int64_t m = 0;
+    for (int64_t i = 0; i < n; ++i)
+        if (start[i]) { off_out[m] = i; seg_alive_out[m] = alive[i]; ++m; }
+    off_out[m] = n;
+    return m;
+}

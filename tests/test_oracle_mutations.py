@@ -88,6 +88,24 @@ MUTATIONS = {
     "priority: ratio not clipped":
         ("double p = w_td * fabs(td_delta[t]) + w_rho * fmin(rho, rho_clip) + w_ent * H;",
          "double p = w_td * fabs(td_delta[t]) + w_rho * rho + w_ent * H;"),
+    "ring: a trajectory that does not fit at the end is squeezed in there instead of starting at slot 0":
+        ("            h = 0;\n        }\n        /* every stored trajectory", "            h = n - T;\n        }\n        /* every stored trajectory"),
+    "ring: the remainder of an evicted trajectory keeps its mass":
+        ("for (int64_t t = s; t < e; ++t) { alive[t] = 0; q[t] = 0u; }", "for (int64_t t = s; t < e; ++t) { alive[t] = 0; }"),
+    "ring: only the overwritten rows of an evicted trajectory die":
+        ("    while (!start[s]) --s;             /* first slot of the trajectory that owns slot i */\n    while (e < n && !start[e]) ++e;",
+         "    while (e < n && 0) ++e;"),
+    "ring: what follows a new trajectory is not split off":
+        ("if (h + T < n) start[h + T] = 1;", ";"),
+    "ring: the slots retired at the end of the buffer keep their trajectories":
+        ("for (int64_t i = h; i < n; ++i) ring_kill_trajectory_at(n, q, alive, start, i);\n            for (int64_t i = h; i < n; ++i) start[i] = (i == h);",
+         "for (int64_t i = h; i < n; ++i) start[i] = (i == h);"),
+    "ring: the write index does not come back to 0 after the last slot":
+        ("*head = h % n;", "*head = h;"),
+    "ring: the slots retired at the end are not counted, so a call may overwrite its own trajectories":
+        ("if (h + T > n) { advance += n - h; h = 0; }", "if (h + T > n) { h = 0; }"),
+    "ring: rows are taken from the start of the call's rows for every trajectory":
+        ("field[f][h + i] = new_field[f][new_off[j] + i];", "field[f][h + i] = new_field[f][i];"),
     "trajectory range ends at its own start offset":
         ("end[j] = off[idx[j] + 1];", "end[j] = off[idx[j]];"),
 }

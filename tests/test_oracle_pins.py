@@ -522,3 +522,160 @@ def test_no_draw_returns_a_filtered_transition_and_the_rest_keep_their_proportio
     u = np.array([((y << 64) + total - 1) // total for y in range(total)], dtype=np.uint64)
     hits = np.bincount(oracle.sample_linear(q, u), minlength=9)
     np.testing.assert_array_equal(hits, q)
+
+
+# ------------------------------------------- circular buffer of trajectories ---
+def _ring_ingest(ring, lens, tag):
+    """Ingest trajectories of the given lengths; row value = tag * 1000 + position in the call, mass = 1 + that."""
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    rows = tag * 1000.0 + np.arange(off[-1], dtype=np.float64)
+    q = (1 + tag * 1000 + np.arange(off[-1])).astype(np.uint32)
+    return ring.ingest(off, [rows, -rows], q), off, rows, q
+
+
+def test_ring_hand_case_with_wrap_around():
+    # capacity 10.  A (4 rows) and B (3 rows) fill slots 0..6.  C (4 rows) does not fit into slots 7..9:
+    # they are retired, C goes to slots 0..3 and evicts A.
+    ring = oracle.Ring(10, 2)
+    ok, _, _, _ = _ring_ingest(ring, [4, 3], 1)
+    assert ok and ring.head == 7
+    assert ring.alive.tolist() == [1] * 7 + [0] * 3
+    assert ring.start.tolist() == [1, 0, 0, 0, 1, 0, 0, 1, 0, 0]
+    assert ring.q.tolist() == [1001, 1002, 1003, 1004, 1005, 1006, 1007, 0, 0, 0]
+    ok, _, _, _ = _ring_ingest(ring, [4], 2)
+    assert ok and ring.head == 4
+    assert ring.alive.tolist() == [1] * 7 + [0] * 3
+    assert ring.start.tolist() == [1, 0, 0, 0, 1, 0, 0, 1, 0, 0]
+    assert ring.q.tolist() == [2001, 2002, 2003, 2004, 1005, 1006, 1007, 0, 0, 0]
+    assert ring.fields[0].tolist() == [2000, 2001, 2002, 2003, 1004, 1005, 1006, 0, 0, 0]
+    assert ring.fields[1].tolist() == [-2000, -2001, -2002, -2003, -1004, -1005, -1006, 0, 0, 0]
+    off, alive = ring.segments()
+    assert off.tolist() == [0, 4, 7, 10] and alive.tolist() == [1, 1, 0]
+
+
+def test_ring_a_trajectory_cut_by_the_write_index_goes_as_a_whole():
+    # A = slots 0..5, B = slots 6..9, head back at 0.  A 2-row trajectory overwrites slots 0..1: A lost
+    # rows, so its slots 2..5 are dead (mass 0) although nothing was written there; B is untouched.
+    ring = oracle.Ring(10, 2)
+    assert _ring_ingest(ring, [6, 4], 1)[0] and ring.head == 0
+    assert _ring_ingest(ring, [2], 2)[0] and ring.head == 2
+    assert ring.alive.tolist() == [1, 1, 0, 0, 0, 0, 1, 1, 1, 1]
+    assert ring.q.tolist() == [2001, 2002, 0, 0, 0, 0, 1007, 1008, 1009, 1010]
+    assert ring.start.tolist() == [1, 0, 1, 0, 0, 0, 1, 0, 0, 0]
+    assert ring.fields[0][2:6].tolist() == [1002, 1003, 1004, 1005]      # stale rows stay, but are dead
+    off, alive = ring.segments()
+    assert off.tolist() == [0, 2, 6, 10] and alive.tolist() == [1, 0, 1]
+    # a trajectory landing in the middle of B's slots cuts B on both sides
+    ring = oracle.Ring(10, 2)
+    assert _ring_ingest(ring, [2, 8], 1)[0]
+    ring.head = 4
+    assert _ring_ingest(ring, [3], 2)[0] and ring.head == 7
+    assert ring.alive.tolist() == [1, 1, 0, 0, 1, 1, 1, 0, 0, 0]
+    assert ring.start.tolist() == [1, 0, 1, 0, 1, 0, 0, 1, 0, 0]
+    assert ring.q.tolist() == [1001, 1002, 0, 0, 2001, 2002, 2003, 0, 0, 0]
+
+
+def test_ring_capacity_exactly_filled_and_refusals():
+    ring = oracle.Ring(8, 2)
+    assert _ring_ingest(ring, [3, 0, 5], 1)[0]                       # an empty trajectory stores nothing
+    assert ring.head == 0 and ring.alive.all()
+    assert ring.start.tolist() == [1, 0, 0, 1, 0, 0, 0, 0]
+    assert _ring_ingest(ring, [8], 2)[0] and ring.head == 0          # one trajectory as long as the buffer
+    assert ring.alive.all() and ring.start.tolist() == [1] + [0] * 7
+    assert ring.q.tolist() == list(range(2001, 2009))
+    before = (ring.q.copy(), ring.alive.copy(), ring.start.copy(), ring.fields[0].copy(), ring.head)
+    assert not _ring_ingest(ring, [9], 3)[0]                         # longer than the buffer
+    assert not _ring_ingest(ring, [5, 5], 3)[0]                      # would overwrite its own first trajectory
+    ring.head = 5
+    assert not _ring_ingest(ring, [2, 4, 2], 3)[0]                   # 8 rows fit, but 2 + 1 retired + 4 + 2 > 8
+    ring.head = 0
+    assert not ring.ingest([0, 3, 2], [np.zeros(3), np.zeros(3)], np.ones(3))   # offsets decrease
+    assert not ring.ingest([1, 3], [np.zeros(3), np.zeros(3)], np.ones(3))      # offsets do not start at 0
+    for a, b in zip(before, (ring.q, ring.alive, ring.start, ring.fields[0], ring.head)):
+        assert np.array_equal(a, b)                                  # a refused call changes nothing
+    ring.head = 5
+    assert _ring_ingest(ring, [2, 4], 3)[0] and ring.head == 4       # 2 + 1 retired + 4 = 7 <= 8
+    assert ring.alive.tolist() == [1, 1, 1, 1, 0, 1, 1, 0]
+    assert ring.start.tolist() == [1, 0, 0, 0, 1, 1, 0, 1]
+
+
+class _ListRing:
+    """The same buffer kept as a list of stored trajectories (an independent formulation: no flags)."""
+
+    def __init__(self, n):
+        self.n, self.head, self.trajs = n, 0, []       # trajs: (first slot, length, tag, first row of the call)
+
+    def _drop_overlapping(self, a, b):
+        self.trajs = [t for t in self.trajs if t[0] + t[1] <= a or t[0] >= b]
+
+    def ingest(self, lens, tag):
+        row = 0
+        for T in lens:
+            if T == 0:
+                continue
+            if self.head + T > self.n:
+                self._drop_overlapping(self.head, self.n)
+                self.head = 0
+            self._drop_overlapping(self.head, self.head + T)
+            self.trajs.append((self.head, T, tag, row))
+            self.head = (self.head + T) % self.n
+            row += T
+
+
+def test_ring_against_a_list_of_trajectories_and_brute_force_draws():
+    rng = np.random.default_rng(31)
+    n = 97
+    ring, model = oracle.Ring(n, 2), _ListRing(n)
+    for call in range(1, 60):
+        lens = rng.integers(0, 14, size=int(rng.integers(1, 6))).tolist()
+        if call % 9 == 0:
+            lens = [int(rng.integers(40, 60))]                         # now and then a long one
+        ok, off, rows, q = _ring_ingest(ring, lens, call)
+        assert ok
+        model.ingest(lens, call)
+        assert ring.head == model.head
+        want_alive = np.zeros(n, dtype=np.uint8)
+        want_q = np.zeros(n, dtype=np.uint32)
+        for (s, T, tag, row) in model.trajs:
+            want_alive[s:s + T] = 1
+            want_q[s:s + T] = 1 + tag * 1000 + row + np.arange(T)
+            np.testing.assert_array_equal(ring.fields[0][s:s + T], tag * 1000.0 + row + np.arange(T))
+            np.testing.assert_array_equal(ring.fields[1][s:s + T], -(tag * 1000.0 + row + np.arange(T)))
+        np.testing.assert_array_equal(ring.alive, want_alive)
+        np.testing.assert_array_equal(ring.q, want_q)                  # dead slots carry no mass
+        seg_off, seg_alive = ring.segments()
+        assert seg_off[0] == 0 and seg_off[-1] == n and np.all(np.diff(seg_off) > 0)
+        live = sorted((s, s + T) for (s, T, _, _) in model.trajs)
+        assert live == [(int(seg_off[j]), int(seg_off[j + 1])) for j in range(len(seg_alive)) if seg_alive[j]]
+        for j in range(len(seg_alive)):                                # segments are all alive or all dead
+            assert ring.alive[seg_off[j]:seg_off[j + 1]].min() == ring.alive[seg_off[j]:seg_off[j + 1]].max()
+    # every threshold by brute force: slot i is drawn exactly q_i times, an evicted slot never
+    total = int(ring.q.sum(dtype=np.uint64))
+    u = np.array([((y << 64) + total - 1) // total for y in range(0, total, 7)], dtype=np.uint64)
+    drawn = oracle.sample_linear(ring.q, u)
+    assert ring.alive[drawn].all()
+    C = np.cumsum(ring.q.astype(np.uint64))
+    np.testing.assert_array_equal(drawn, np.searchsorted(C, np.arange(0, total, 7, dtype=np.uint64), side="right"))
+
+
+def test_ring_retrace_over_the_segments_equals_retrace_per_live_trajectory():
+    # the CSR view of a wrapped buffer goes through Retrace like any other batch: a live trajectory's
+    # targets do not depend on what lies around it (dead stretches included)
+    rng = np.random.default_rng(32)
+    n = 211
+    ring = oracle.Ring(n, 4)                                           # r, V, log pi, log mu
+    stored = {}
+    for call in range(25):
+        lens = rng.integers(1, 30, size=3)
+        off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+        T = int(off[-1])
+        new = [rng.normal(0, 1, T), rng.random(T), rng.normal(-3, 1, T), rng.normal(-3, 1, T)]
+        assert ring.ingest(off, new, rng.integers(1, 99, T))
+    seg_off, seg_alive = ring.segments()
+    assert seg_alive.any() and not seg_alive.all()                     # wrapped: some stretches are dead
+    vt, adv, dl = oracle.retrace(seg_off, *ring.fields, 0.97, 0.9)
+    for j in np.flatnonzero(seg_alive):
+        a, b = int(seg_off[j]), int(seg_off[j + 1])
+        one = oracle.retrace([0, b - a], *[f[a:b] for f in ring.fields], 0.97, 0.9)
+        np.testing.assert_array_equal(vt[a:b], one[0])
+        np.testing.assert_array_equal(adv[a:b], one[1])
