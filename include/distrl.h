@@ -258,6 +258,73 @@ int distrl_update_priorities(distrl_sampler *s, const int64_t *idx, int64_t k,
 int distrl_replay_overwrite(distrl_sampler *s, int64_t head, int64_t k, const uint32_t *new_q,
                             void *stream);
 
+/* ---------------------------------------------------------------------------
+ * Circular replay buffer of whole trajectories (App. A "Circular Replay Buffer":
+ * capacity N, the write index advances as i <- (i+1) mod N and new experiences
+ * overwrite the oldest; Section 5.3 prioritises and replays trajectories).
+ *
+ * The buffer is the caller's SoA arrays of N slots (any fp32 per-transition
+ * fields: rewards, values, log-probs, entropy, ...) and the masses prio_q.  The
+ * library keeps its structure and, after every ingest, hands back the CSR view
+ * the other entry points take:
+ *   traj_offsets[0 .. m_capacity] : segment offsets; the flat buffer is cut into
+ *       segments, each a live trajectory or a dead stretch; entries past the
+ *       last segment are N (empty segments), so a call that takes traj_offsets
+ *       may always be given n_trajectories = m_capacity;
+ *   traj_alive[0 .. m_capacity)   : 1.0f for a live trajectory, 0.0f otherwise
+ *       (a score for distrl_filter_trajectories with threshold 0.5, which
+ *       zeroes the masses of dead stretches after priorities were recomputed
+ *       for the whole buffer).
+ * Rules of an ingest, trajectory by trajectory in the order given:
+ *   - a trajectory occupies consecutive slots from the write index on (the
+ *     recursion of Section 5.2 runs along it); one that would reach past slot
+ *     N-1 starts at slot 0 instead and the slots left at the end are retired;
+ *   - every stored trajectory that loses a slot is evicted as a whole: its
+ *     remaining slots are dead and their masses 0, so no draw returns them
+ *     (their rows stay in place until overwritten);
+ *   - an empty trajectory stores nothing.
+ * A call whose rows plus retired slots exceed N (it would overwrite its own
+ * trajectories) is refused with DISTRL_ERR_SIZE and changes nothing: ingest in
+ * smaller batches.  Masses of new rows come from the caller (e.g. Retrace and
+ * priorities run on the new batch first); with a sampler over prio_q given,
+ * every partial sum is repaired exactly, as if the sampler had been rebuilt.
+ * ------------------------------------------------------------------------- */
+typedef struct distrl_replay distrl_replay; /* small host-side handle */
+#define DISTRL_REPLAY_MAX_FIELDS 8
+
+size_t distrl_replay_workspace_bytes(int64_t capacity);
+
+/*  fields : HOST array of n_fields (<= DISTRL_REPLAY_MAX_FIELDS) device arrays of
+ *      `capacity` floats each; prio_q : [capacity]; traj_offsets : [m_capacity+1];
+ *      traj_alive : [m_capacity].  All are zero-filled / initialised to the empty
+ *      buffer (one dead segment, no mass) on `stream`; dead rows stay finite.
+ *  workspace : >= distrl_replay_workspace_bytes(capacity), 256-byte aligned; its
+ *      first word is a status word for distrl_get_status (DISTRL_ERR_SIZE: more
+ *      segments than m_capacity; DISTRL_ERR_OFFSETS: see distrl_replay_ingest).
+ *  The handle keeps the pointers; free it with distrl_replay_destroy (that frees
+ *  no device memory).  All calls on one buffer go to one stream. */
+int distrl_replay_create(int64_t capacity, int n_fields, float *const *fields, uint32_t *prio_q,
+                         int64_t *traj_offsets, float *traj_alive, int64_t m_capacity,
+                         void *workspace, size_t workspace_bytes, void *stream, distrl_replay **out);
+
+/*  k new trajectories whose rows are concatenated in new_fields / new_q:
+ *  new_offsets_host : HOST array [k+1], non-decreasing from 0 (the learner knows
+ *      the lengths of what it received); new_offsets : the same values on the
+ *      DEVICE (the batch's own traj_offsets); a mismatch is reported as
+ *      DISTRL_ERR_OFFSETS in the status word and leaves the structure unspecified.
+ *  new_fields : HOST array of n_fields device arrays of new_offsets_host[k] rows;
+ *  new_q : device masses of those rows, each in [1, 2^32-1].
+ *  sampler : a sampler built over this buffer's prio_q, or NULL (then only
+ *      prio_q is written and the caller rebuilds its sampler).
+ *  n_segments_out_device : device int64 or NULL; receives the number of segments. */
+int distrl_replay_ingest(distrl_replay *rb, distrl_sampler *sampler, int64_t k,
+                         const int64_t *new_offsets_host, const int64_t *new_offsets,
+                         const float *const *new_fields, const uint32_t *new_q,
+                         int64_t *n_segments_out_device, void *stream);
+
+int64_t distrl_replay_head(const distrl_replay *rb); /* next write index; -1 for NULL */
+int distrl_replay_destroy(distrl_replay *rb);
+
 /*
  * Retrace targets (Section 5.2), priorities (Section 5.3) and the sampler's sum
  * tree in ONE pass over the trajectory buffer: what distrl_retrace_targets,
@@ -321,7 +388,9 @@ int distrl_trajectory_ranges(int64_t m, const int64_t *traj_offsets, const int64
  * the transitions stay where they are until overwritten.  Masses of retained
  * trajectories are left as they are.  Call it between distrl_compute_priorities
  * and distrl_build_sampler (or rebuild the sampler afterwards); at least one
- * retained trajectory must have a transition, or there is nothing to draw.
+ * retained trajectory must have a transition, or there is nothing to draw
+ * (distrl_sample then returns index -1 and weight 0 for every draw and records
+ * DISTRL_ERR_INDEX in the sampler's status word).
  *   traj_score : [M] device scores (e.g. V_traj's outputs);  prio_q : [N] in/out.
  *   kept_out_device : device uint64 or NULL; receives the number retained.
  */

@@ -6,5 +6,5 @@ The product is the C-ABI CUDA library under ``csrc/`` (declared in
 benchmarks.  There is no CPU path.
 """
 from .binding import *  # noqa: F401,F403
-from .binding import (DistrlError, Sampler, alloc_workspace, distrl_batch, distrl_prio_cfg, library_path,
+from .binding import (DistrlError, Replay, Sampler, alloc_workspace, distrl_batch, distrl_prio_cfg, library_path,
                       make_batch, make_prio_cfg)

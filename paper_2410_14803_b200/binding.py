@@ -82,6 +82,11 @@ def _load():
                                                  ctypes.POINTER(distrl_prio_cfg), vp, vp, vp, vp, vp, vp, sz, vp, sz, vp,
                                                  ctypes.POINTER(vp)]),
         "distrl_replay_overwrite": (ci, [vp, i64, i64, vp, vp]),
+        "distrl_replay_workspace_bytes": (sz, [i64]),
+        "distrl_replay_create": (ci, [i64, ci, vp, vp, vp, vp, i64, vp, sz, vp, ctypes.POINTER(vp)]),
+        "distrl_replay_ingest": (ci, [vp, vp, i64, vp, vp, vp, vp, vp, vp]),
+        "distrl_replay_head": (i64, [vp]),
+        "distrl_replay_destroy": (ci, [vp]),
         "distrl_actor_coefficients": (ci, [i64, vp, i64, vp, vp, vp, vp, vp, vp, vp]),
         "distrl_trajectory_ranges": (ci, [i64, vp, vp, i64, vp, vp, vp, vp]),
         "distrl_filter_trajectories": (ci, [i64, i64, vp, vp, f32, vp, vp, vp]),
@@ -345,6 +350,76 @@ def distrl_filter_trajectories(traj_offsets: torch.Tensor, traj_score: torch.Ten
                                               _ptr(traj_score, torch.float32), threshold, _ptr(prio_q),
                                               _ptr(kept_out, torch.int64), _stream(stream)),
            "distrl_filter_trajectories")
+
+
+class Replay:
+    """Owns the host handle of a circular buffer of trajectories and keeps its tensors alive."""
+
+    def __init__(self, handle, fields, prio_q, traj_offsets, traj_alive, workspace):
+        self.handle = handle
+        self.fields, self.prio_q = fields, prio_q
+        self.traj_offsets, self.traj_alive, self.workspace = traj_offsets, traj_alive, workspace
+
+    @property
+    def head(self) -> int:
+        return int(_load().distrl_replay_head(self.handle))
+
+    def close(self):
+        if self.handle:
+            _load().distrl_replay_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def distrl_replay_workspace_bytes(capacity: int) -> int:
+    return int(_load().distrl_replay_workspace_bytes(capacity))
+
+
+def _ptr_array(tensors, dtype):
+    arr = (ctypes.c_void_p * max(len(tensors), 1))()
+    for i, t in enumerate(tensors):
+        arr[i] = _ptr(t, dtype)
+    return arr
+
+
+def distrl_replay_create(fields, prio_q: torch.Tensor, traj_offsets: torch.Tensor, traj_alive: torch.Tensor,
+                         workspace: torch.Tensor, stream=None) -> Replay:
+    """fields: list of fp32 CUDA tensors of `capacity` elements each (the buffer's SoA arrays)."""
+    if prio_q.element_size() != 4:
+        raise ValueError("prio_q must hold 32-bit masses")
+    capacity = prio_q.numel()
+    for f in fields:
+        if f.numel() != capacity:
+            raise ValueError("every field needs `capacity` elements")
+    if traj_offsets.numel() != traj_alive.numel() + 1:
+        raise ValueError("traj_offsets needs one more entry than traj_alive")
+    out = ctypes.c_void_p()
+    _check(_load().distrl_replay_create(capacity, len(fields), _ptr_array(fields, torch.float32), _ptr(prio_q),
+                                        _ptr(traj_offsets, torch.int64), _ptr(traj_alive, torch.float32),
+                                        traj_alive.numel(), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream(stream),
+                                        ctypes.byref(out)), "distrl_replay_create")
+    return Replay(out.value, list(fields), prio_q, traj_offsets, traj_alive, workspace)
+
+
+def distrl_replay_ingest(rb: Replay, sampler: Optional[Sampler], new_offsets_host, new_offsets: torch.Tensor, new_fields,
+                         new_q: torch.Tensor, n_segments_out: Optional[torch.Tensor] = None, stream=None):
+    """new_offsets_host: host int64 array (numpy) [k+1]; new_offsets: the same on the device."""
+    import numpy as np
+    host = np.ascontiguousarray(new_offsets_host, dtype=np.int64)
+    if new_offsets.numel() != host.shape[0]:
+        raise ValueError("host and device offsets differ in length")
+    if len(new_fields) != len(rb.fields):
+        raise ValueError("one array of new rows per field")
+    _check(_load().distrl_replay_ingest(rb.handle, sampler.handle if sampler is not None else None, host.shape[0] - 1,
+                                        host.ctypes.data_as(ctypes.c_void_p), _ptr(new_offsets, torch.int64),
+                                        _ptr_array(new_fields, torch.float32), _ptr(new_q),
+                                        _ptr(n_segments_out, torch.int64), _stream(stream)), "distrl_replay_ingest")
 
 
 def distrl_sampler_total(s: Sampler, total_out: torch.Tensor, stream=None):

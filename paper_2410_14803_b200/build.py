@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libdistrl_b200.so")
-SOURCES = ["api.cu", "retrace.cu", "priority.cu", "sampler.cu", "batch.cu"]
+SOURCES = ["api.cu", "retrace.cu", "priority.cu", "sampler.cu", "batch.cu", "replay.cu"]
 
 
 def _newest_source_mtime() -> float:
@@ -26,7 +26,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB_PATH + ".tmp.%d" % os.getpid()
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC, "-o", tmp]
+           "-shared", "-Xcompiler", "-fPIC", "-t", "0", "-I", INCLUDE, "-I", CSRC, "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += os.environ.get("DISTRL_NVCC_EXTRA", "").split()   # e.g. -D overrides of tuning constants

@@ -198,6 +198,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     __shared__ __align__(8) uint64_t s_bar;
     __shared__ int s_last;
     __shared__ unsigned int s_qmin; // smallest mass drawn by this block
+    __shared__ int s_nothing;       // the total mass is zero: no draw is possible (the same in every block)
     const int lane = threadIdx.x & 31;
     grid_dependency_wait();
     grid_launch_dependents();
@@ -205,6 +206,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     // them); sizes are rounded up to 16 bytes, the slack lies inside the levels' 256-byte padding.
     if (threadIdx.x == 0) {
         s_qmin = 0xffffffffu;
+        s_nothing = 0;
         mbar_init(&s_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         unsigned int bytes = 0;
@@ -236,6 +238,17 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
         const unsigned long long total = __shfl_sync(0xffffffffu, incl, 31);
         unsigned long long y = __umul64hi(uj, total);
         int64_t node = 0;
+        if (total == 0ull) { // every mass is zero (an empty or fully filtered buffer): there is nothing to draw
+            if (lane == 0) {
+                set_status(&t.hdr->status, DISTRL_ERR_INDEX);
+                s_nothing = 1;
+                idx_out[j] = -1;
+                if (w_out) {
+                    w_out[j] = 0.f;
+                    if (normalise && together) { my_q = 0xffffffffu; mine = true; }
+                }
+            }
+        } else {
         while (true) {
             int c = pick_lane(incl, v, y);
             y -= __shfl_sync(0xffffffffu, incl - v, c);
@@ -278,6 +291,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
                 }
             }
         }
+        }
     }
     if (!(w_out && normalise)) return;
     if (together) {
@@ -301,7 +315,7 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
             s_qmin = __ldcg(&t.hdr->qmin);
         }
         __syncthreads();
-        if (mine) w_out[j] = powf((float)((double)my_q / (double)s_qmin), -beta);
+        if (mine) w_out[j] = s_nothing ? 0.f : powf((float)((double)my_q / (double)s_qmin), -beta);
         if (threadIdx.x == 0) {
             const unsigned int gone = atomicAdd(&t.hdr->left, 1u);
             if (gone == gridDim.x - 1) { // everybody has read the minimum: ready for the next call
@@ -325,6 +339,10 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     }
     __syncthreads();
     if (!s_last) return;
+    if (s_nothing) { // nothing was drawn: the weights stay 0
+        if (threadIdx.x == 0) t.hdr->done = 0u;
+        return;
+    }
     // Up to kTailKeep parked masses per thread stay in registers between the search for the minimum and
     // the rescaling (a batch of 4096 draws is read once); longer batches are read again.
     constexpr int kTailKeep = 8;
@@ -558,19 +576,17 @@ __global__ void __launch_bounds__(kSmallThreads) update_small_kernel(
 // touched leaf group stores them, recomputes the group's sum from the masses themselves and adds the
 // difference to every ancestor, so the tree again equals a rebuild.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) overwrite_kernel(Tree t, int64_t a, int64_t b, const uint32_t *__restrict__ src) {
-    grid_dependency_wait();
-    grid_launch_dependents();
-    const int lane = threadIdx.x & 31;
-    const int64_t g = a / kLeaf + (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
-    if (g > (b - 1) / kLeaf) return; // warp-uniform
+// One leaf group of the overwrite: slots of [a, b) inside group g receive src[i - a] (src null: 0), the
+// group's sum is recomputed from the masses themselves and the difference goes to every ancestor.
+__device__ __forceinline__ void overwrite_group(const Tree &t, int64_t g, int64_t a, int64_t b,
+                                                const uint32_t *__restrict__ src, int lane) {
     unsigned long long sum = 0;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
         const int64_t i = g * kLeaf + 4 * lane + e;
         uint32_t v = 0u;
         if (i < t.n) {
-            if (i >= a && i < b) { v = src[i - a]; t.q[i] = v; }
+            if (i >= a && i < b) { v = src ? src[i - a] : 0u; t.q[i] = v; }
             else v = __ldcg(t.q + i);
         }
         sum += v;
@@ -578,7 +594,7 @@ __global__ void __launch_bounds__(256) overwrite_kernel(Tree t, int64_t a, int64
     sum = warp_sum_u64(sum);
     if (lane == 0) {
         const unsigned long long old = t.lvl[1][g];
-        t.lvl[1][g] = sum; // this warp is the only writer of the group in this launch
+        t.lvl[1][g] = sum; // this warp is the only writer of the group at this time
         const unsigned long long diff = sum - old; // mod 2^64
         if (diff) {
             int64_t node = g / kFan;
@@ -588,6 +604,28 @@ __global__ void __launch_bounds__(256) overwrite_kernel(Tree t, int64_t a, int64
             }
         }
     }
+}
+
+__global__ void __launch_bounds__(256) overwrite_kernel(Tree t, int64_t a, int64_t b, const uint32_t *__restrict__ src) {
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const int lane = threadIdx.x & 31;
+    const int64_t g = a / kLeaf + (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    if (g > (b - 1) / kLeaf) return; // warp-uniform
+    overwrite_group(t, g, a, b, src, lane);
+}
+
+// Zero masses for a range of slots that only the device knows (range[0] .. range[1]; empty when
+// end <= begin): one block, its warps striding over the leaf groups.
+__global__ void __launch_bounds__(256) zero_range_kernel(Tree t, const int64_t *__restrict__ range) {
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int64_t a = range[0], b = range[1];
+    if (a < 0) a = 0;
+    if (b > t.n) b = t.n;
+    if (b <= a) return;
+    for (int64_t g = a / kLeaf + warp; g <= (b - 1) / kLeaf; g += 8) overwrite_group(t, g, a, b, nullptr, lane);
 }
 
 } // namespace distrl
@@ -655,6 +693,22 @@ int sampler_build_upper(const distrl_sampler *s, cudaStream_t st) {
     if (s->tree.levels >= 3) {
         DISTRL_CUDA_TRY(launch_pdl(build_upper_kernel, dim3(1), dim3(1024), 0, st, s->tree));
     }
+    return DISTRL_OK;
+}
+
+int64_t sampler_size(const distrl_sampler *s) { return s->tree.n; }
+const uint32_t *sampler_masses(const distrl_sampler *s) { return s->tree.q; }
+
+int sampler_overwrite_run(distrl_sampler *s, int64_t a, int64_t b, const uint32_t *src, cudaStream_t st) {
+    if (b <= a) return DISTRL_OK;
+    const int64_t groups = (b - 1) / kLeaf - a / kLeaf + 1;
+    DISTRL_CUDA_TRY(launch_pdl(overwrite_kernel, dim3((unsigned)ceil_div(groups * 32, 256)), dim3(256), 0, st, s->tree,
+                               a, b, src));
+    return DISTRL_OK;
+}
+
+int sampler_zero_range(distrl_sampler *s, const int64_t *range_device, cudaStream_t st) {
+    DISTRL_CUDA_TRY(launch_pdl(zero_range_kernel, dim3(1), dim3(256), 0, st, s->tree, range_device));
     return DISTRL_OK;
 }
 
@@ -779,11 +833,8 @@ extern "C" int distrl_replay_overwrite(distrl_sampler *s, int64_t head, int64_t 
     const int64_t first = (head + k <= n) ? k : n - head;
     const int64_t runs[2][3] = {{head, head + first, 0}, {0, k - first, first}};
     for (int r = 0; r < 2; ++r) {
-        const int64_t a = runs[r][0], b = runs[r][1];
-        if (b <= a) continue;
-        const int64_t groups = (b - 1) / kLeaf - a / kLeaf + 1;
-        DISTRL_CUDA_TRY(launch_pdl(overwrite_kernel, dim3((unsigned)ceil_div(groups * 32, 256)), dim3(256), 0, st,
-                                   s->tree, a, b, new_q + runs[r][2]));
+        const int rc = sampler_overwrite_run(s, runs[r][0], runs[r][1], new_q + runs[r][2], st);
+        if (rc) return rc;
     }
     return DISTRL_OK;
 }

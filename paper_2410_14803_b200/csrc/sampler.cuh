@@ -21,4 +21,12 @@ void sampler_tree_base(const distrl_sampler *s, TreeBase *out);
 // Levels 3 and above from level 2 (a no-op for trees of one or two levels).
 int sampler_build_upper(const distrl_sampler *s, cudaStream_t st);
 
+// What the circular buffer of trajectories needs: the masses of the slots [a, b) replaced by
+// src[0 .. b-a) (src null: by zeros), and zeros for a range that only the device knows
+// (range_device: int64[2] = begin, end); every partial sum of the tree repaired exactly.
+int64_t sampler_size(const distrl_sampler *s);
+const uint32_t *sampler_masses(const distrl_sampler *s);
+int sampler_overwrite_run(distrl_sampler *s, int64_t a, int64_t b, const uint32_t *src, cudaStream_t st);
+int sampler_zero_range(distrl_sampler *s, const int64_t *range_device, cudaStream_t st);
+
 } // namespace distrl

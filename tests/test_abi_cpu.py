@@ -89,6 +89,16 @@ def test_argument_validation_happens_before_any_device_work():
     assert lib.distrl_update_priorities(None, None, 1, None, None, None, None, ctypes.byref(cfg), None, None) \
         == binding.ERR_NULL
     assert lib.distrl_destroy_sampler(None) == 0
+    # circular buffer of trajectories
+    rb = ctypes.c_void_p()
+    assert lib.distrl_replay_create(0, 0, None, None, None, None, 1, None, 0, None, ctypes.byref(rb)) == binding.ERR_SIZE
+    assert lib.distrl_replay_create(8, 9, None, None, None, None, 1, None, 0, None, ctypes.byref(rb)) == binding.ERR_SIZE
+    assert lib.distrl_replay_create(8, 0, None, None, None, None, 1, None, 0, None, ctypes.byref(rb)) == binding.ERR_NULL
+    assert lib.distrl_replay_create(8, 0, None, None, None, None, 1, None, 0, None, None) == binding.ERR_NULL
+    assert lib.distrl_replay_ingest(None, None, 1, None, None, None, None, None, None) == binding.ERR_NULL
+    assert lib.distrl_replay_head(None) == -1 and lib.distrl_replay_destroy(None) == 0
+    assert distrl.distrl_replay_workspace_bytes(1 << 24) == 256 + 2 * (1 << 21) + 256 * ((513 * 8 + 255) // 256)
+    assert lib.distrl_set_cooperative_launch(1) == 1
 
 
 def test_binding_refuses_host_tensors():
