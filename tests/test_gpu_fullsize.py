@@ -1,5 +1,6 @@
-"""Full-size parity cases: the workloads at their real sizes, checked on sampled trajectories that the
-oracle evaluates one by one, plus properties that hold at any size."""
+"""Full-size parity cases: the workloads at their real sizes.  The token-level workload is checked twice:
+quickly on sampled trajectories that the oracle evaluates one by one plus properties that hold at any
+size, and once on every step (the slow test of this file)."""
 import numpy as np
 import pytest
 import torch
@@ -93,6 +94,104 @@ def test_token_level_full_size_sampled_trajectories():
     s.close()
 
 
+def test_token_level_full_size_every_step():
+    # All 67,108,864 steps against the oracle (about 45 s on a B200 machine, most of it the oracle's own
+    # token sums over 1.1e9 tokens).  The oracle runs over ranges of whole trajectories, so the widened
+    # fp64 copies of the token arrays stay at a few hundred MB at a time.
+    w = synth.make_workload(4)
+    a = w.arrays
+    n, off, sto = w.n, a["traj_offsets"], a["step_token_offsets"]
+    t_off, t_r, t_V, t_sto = dev(off), dev(a["rewards"]), dev(a["values"]), dev(sto)
+    t_tp = dev(a["tok_logp_target"], torch.bfloat16)
+    t_tm = dev(a["tok_logp_behaviour"], torch.bfloat16)
+    batch = distrl.make_batch(t_off, t_r, t_V, None, None, None, t_sto, t_tp, t_tm)
+    out = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(5)]
+    ws = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws)
+    distrl.distrl_retrace_targets(batch, w.gamma, w.lam, *out, workspace=ws)
+    assert distrl.distrl_get_status(ws) == 0
+    del t_tp, t_tm, batch
+    vt, adv, dl, lpo, lmo = (o.cpu().numpy() for o in out)
+    m = off.shape[0] - 1
+    step = 1 << 18                                           # trajectories per range (about 4 M steps, 67 M tokens)
+    for j0 in range(0, m, step):
+        j1 = min(m, j0 + step)
+        s0, s1 = int(off[j0]), int(off[j1])
+        k0, k1 = int(sto[s0]), int(sto[s1])
+        sub_sto = sto[s0:s1 + 1] - k0
+        lp = oracle.token_logp(sub_sto, oracle.bf16_bits_to_f64(a["tok_logp_target"][k0:k1]))
+        lm = oracle.token_logp(sub_sto, oracle.bf16_bits_to_f64(a["tok_logp_behaviour"][k0:k1]))
+        o_vt, o_adv, o_dl = oracle.retrace(off[j0:j1 + 1] - s0, a["rewards"][s0:s1], a["values"][s0:s1], lp, lm,
+                                           w.gamma, w.lam)
+        where = "trajectories %d..%d: " % (j0, j1)
+        assert_close(lpo[s0:s1], lp, where + "token logp_target")
+        assert_close(lmo[s0:s1], lm, where + "token logp_behaviour")
+        assert_close(vt[s0:s1], o_vt, where + "v_target")
+        assert_close(adv[s0:s1], o_adv, where + "advantage")
+        assert_close(dl[s0:s1], o_dl, where + "td_delta")
+
+
+def test_fused_pass_full_size():
+    # workload 3 at its real size through the one-pass entry point, as the benchmark's fused mode runs it:
+    # every target, mass, fixed-point image and partial sum, then a draw and a refresh on the sampler it built
+    from helpers import prio_cfg_of, read_tree, sample_by_prefix, tree_from_q
+    w = synth.make_workload(3)
+    a = w.arrays
+    n = w.n
+    cfg = prio_cfg_of(w)
+    scale = synth.heavy_tail_scale(w)
+    t = [dev(a["traj_offsets"]), dev(a["rewards"]), dev(a["values"]), dev(a["logp_target"]), dev(a["logp_behaviour"])]
+    t_ent, t_sc = dev(a["entropy"]), dev(scale)
+    vt, adv, dl, mass = (torch.full((n,), float("nan"), dtype=torch.float32, device="cuda") for _ in range(4))
+    tq = torch.zeros(n, dtype=torch.int32, device="cuda")
+    ws_r = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(n))
+    ws_s = distrl.alloc_workspace(distrl.distrl_sampler_workspace_bytes(n))
+    distrl.distrl_workspace_init(ws_r)
+    distrl.distrl_workspace_init(ws_s)
+    s = distrl.distrl_retrace_priorities_build(distrl.make_batch(*t), w.gamma, w.lam, t_ent, t_sc, cfg, vt, adv, dl, tq,
+                                               mass, retrace_workspace=ws_r, sampler_workspace=ws_s)
+    assert distrl.distrl_get_status(ws_r) == 0
+    o_vt, o_adv, o_dl = oracle.retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"],
+                                       a["logp_behaviour"], w.gamma, w.lam)
+    assert_close(vt.cpu().numpy(), o_vt, "v_target")
+    assert_close(adv.cpu().numpy(), o_adv, "advantage")
+    assert_close(dl.cpu().numpy(), o_dl, "td_delta")
+    o_mass = oracle.priority_mass(o_dl * scale.astype(np.float64), a["logp_target"], a["logp_behaviour"], a["entropy"],
+                                  w.w_td, w.w_rho, w.w_ent, w.rho_clip, w.alpha)
+    assert_close(mass.cpu().numpy(), o_mass, "prio_mass")
+    q = tq.cpu().numpy().view(np.uint32)
+    np.testing.assert_array_equal(q, oracle.quantise(mass.cpu().numpy(), w.scale))
+    got, info = read_tree(s)
+    for lvl_got, lvl_want in zip(got, tree_from_q(q, info)):
+        np.testing.assert_array_equal(lvl_got, lvl_want)
+    u = synth.uniforms(w, 0)
+    idx = torch.empty(w.batch, dtype=torch.int64, device="cuda")
+    wts = torch.empty(w.batch, dtype=torch.float32, device="cuda")
+    distrl.distrl_sample(s, dev(u.view(np.int64)), w.beta, True, idx, wts)
+    h_idx = idx.cpu().numpy()
+    np.testing.assert_array_equal(h_idx, sample_by_prefix(q, u))
+    assert_close(wts.cpu().numpy(), oracle.is_weights(q, h_idx, w.beta, True), "is_weight")
+    gm = torch.empty(w.batch, dtype=torch.float32, device="cuda")
+    distrl.distrl_update_priorities(s, idx, dev(synth.fresh_abs_delta(w, 0)), t[3], t[4], t_ent, cfg, gm)
+    oracle.update_from_mass(q, h_idx, gm.cpu().numpy(), w.scale)
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), q)
+    got, info = read_tree(s)
+    for lvl_got, lvl_want in zip(got, tree_from_q(q, info)):
+        np.testing.assert_array_equal(lvl_got, lvl_want)
+    assert distrl.distrl_get_status(ws_s) == 0
+    s.close()
+
+
+def test_bootstrap_values_full_size():
+    # workload 3 at its real size with a bootstrap value per trajectory (the pipelined kernel's BOOT path)
+    from helpers import check_retrace
+    w = synth.make_workload(3)
+    a = w.arrays
+    boot = np.random.default_rng(12).normal(0, 1, w.m).astype(np.float32)
+    check_retrace(a["traj_offsets"], a["rewards"], a["values"], a["logp_target"], a["logp_behaviour"], w.gamma, w.lam,
+                  boot=boot)
+
+
 def test_large_buffer_trajectory_priorities_and_actor_coefficients():
     # workload 3 at its real size (16,777,216 steps, 1.4 M trajectories), every output against the oracle
     from helpers import prio_cfg_of
@@ -118,8 +217,8 @@ def test_large_buffer_trajectory_priorities_and_actor_coefficients():
 
 
 def test_large_buffer_monte_carlo_returns():
-    # workload 3 at its real size: 8192 tiles, more than the persistent grid holds at once, so blocks take
-    # tiles by block number first and by ticket afterwards; every return and label against the oracle
+    # workload 3 at its real size: 8192 tiles, many more than the persistent grid holds at once; every return
+    # and label against the oracle
     w = synth.make_workload(3)
     a = w.arrays
     n = w.n
