@@ -87,6 +87,69 @@ def _oracle_sample(w, budget_transitions=2_000_000, draws=48):
     return est, desc, dict(stream_s_per_transition=t_stream / ns, draw_s=t_draw + t_upd)
 
 
+# ---- all-cores leg: the same oracle routines over contiguous ranges of whole trajectories, one process per core.
+# Worker processes are started with "spawn" (a process forked after the first CUDA call hangs); each loads its
+# range from a file once, untimed, and the timed call only computes.
+_MC = {}
+
+
+def _mc_load(job):
+    path, j0, j1 = job
+    import oracle
+    z = np.load(path)
+    off = z["off"]
+    s0, s1 = int(off[j0]), int(off[j1])
+    _MC["args"] = (off[j0:j1 + 1] - s0, z["r"][s0:s1], z["V"][s0:s1], z["lp"][s0:s1], z["lm"][s0:s1], z["ent"][s0:s1])
+    _MC["oracle"] = oracle
+    oracle.quantise(np.ones(4, dtype=np.float32), 1.0)      # loads the library
+    return s1 - s0
+
+
+def _mc_compute(cfg):
+    gamma, lam, w_td, w_rho, w_ent, rho_clip, alpha, scale = cfg
+    o = _MC["oracle"]
+    off, r, V, lp, lm, ent = _MC["args"]
+    vt, adv, dl = o.retrace(off, r, V, lp, lm, gamma, lam)
+    mass = o.priority_mass(dl, lp, lm, ent, w_td, w_rho, w_ent, rho_clip, alpha)
+    q = o.quantise(mass.astype(np.float32), scale)
+    return int(q[:8].sum())
+
+
+def _oracle_all_cores(w, per_core=1_000_000):
+    """Retrace + priority + quantise (the stages without a dependency between trajectories) on all host cores.
+    Returns (transitions per second, cores, description).  Fixed-N fp32 workloads only."""
+    import multiprocessing as mp
+    import tempfile
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except Exception:
+        cores = os.cpu_count() or 1
+    a = w.arrays
+    off = a["traj_offsets"]
+    ns_want = min(w.n, per_core * cores)
+    j_end = max(cores, int(np.searchsorted(off, ns_want, side="right")) - 1)
+    cuts = [int(np.searchsorted(off, int(off[j_end]) * c // cores, side="left")) for c in range(cores + 1)]
+    cuts[0], cuts[-1] = 0, j_end
+    ns = int(off[j_end])
+    with tempfile.TemporaryDirectory() as d:
+        path = os.path.join(d, "sample.npz")
+        np.savez(path, off=off[:j_end + 1], r=a["rewards"][:ns], V=a["values"][:ns], lp=a["logp_target"][:ns],
+                 lm=a["logp_behaviour"][:ns], ent=a["entropy"][:ns])
+        ctx = mp.get_context("spawn")
+        with ctx.Pool(cores) as pool:
+            jobs = [(path, cuts[c], cuts[c + 1]) for c in range(cores)]
+            pool.map(_mc_load, jobs, chunksize=1)
+            cfg = (w.gamma, w.lam, w.w_td, w.w_rho, w.w_ent, w.rho_clip, w.alpha, w.scale)
+            pool.map(_mc_compute, [cfg] * cores, chunksize=1)          # warm-up
+            t0 = time.perf_counter()
+            pool.map(_mc_compute, [cfg] * cores, chunksize=1)
+            dt = time.perf_counter() - t0
+    desc = ("multi-core baseline: oracle Retrace + priority + quantise (fp64, same routines) over %d contiguous "
+            "ranges of whole trajectories, one process per core, first %d transitions in %.2f s; the sampler stages "
+            "are not in this figure" % (cores, ns, dt))
+    return ns / dt, cores, desc
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -106,8 +169,9 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": METRIC, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": _config(w, args, l2="n/a (CPU)"),
-        "cpu_baseline": {"value": value, "unit": METRIC, "cores": 1, "kind": "oracle", "sample": desc},
+        "config": _config(w, args),
+        "estimated": True,   # scaled from a bounded sample of the workload (see cpu_baseline.sample)
+        "cpu_baseline": {"value": value, "unit": METRIC, "cores": 1, "kind": "oracle", "sample": desc, "estimated": True},
         "e2e": {"value": value, "unit": METRIC, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -115,7 +179,23 @@ def run_reference(args):
     return 0
 
 
-def _config(w, args, l2):
+def _step_bytes(w, args):
+    """Algorithmic bytes of the three streaming stages of one step: (Retrace call, priorities, sampler build)."""
+    n, m = w.n, w.m
+    if w.token_level:   # r, V, step offsets, both bf16 token arrays in; v_target, advantage, td_delta, logpi, logmu out; offsets
+        retrace_bytes = (8 + 8 + 20) * n + 4 * int(w.arrays["step_token_offsets"][-1]) + 8 * (m + 1)
+    else:               # r, V, logpi, logmu in; v_target, advantage, td_delta out; offsets
+        retrace_bytes = 28 * n + 8 * (m + 1)
+    prio_bytes = 20 * n                          # delta, logpi, logmu, entropy in; q out
+    build_bytes = 4 * n + 8 * (n // 128)
+    if getattr(args, "fused", False):   # r, V, logpi, logmu, entropy (+ scale) in; v_target, advantage, q out; offsets; tree levels 1-2
+        retrace_bytes = (20 + (4 if w.heavy_tail else 0) + 12) * n + 8 * (m + 1) + 8 * (n // 128)
+    return retrace_bytes, prio_bytes, build_bytes
+
+
+def _config(w, args):
+    l2 = "inputs larger than L2 (%.0f MB touched per step), two copies of the inputs alternate between steps" % (
+        sum(_step_bytes(w, args)) / 1e6)
     return {"workload": "%s (configs[%d]): N=%d transitions, M=%d trajectories, batch k=%d, %d sample->update rounds"
                         % (w.name, w.index, w.n, w.m, w.batch, w.rounds),
             "gamma": w.gamma, "lambda": w.lam, "alpha": w.alpha, "beta": w.beta, "fixed_point_scale": w.scale,
@@ -246,6 +326,7 @@ def run_ours(args):
             self.d_nd.copy_(host_nd, non_blocking=True)
 
     main_set = InputSet()
+    sets = [main_set, InputSet()]   # two copies of the inputs: consecutive steps never read the same arrays
 
     # The heavy-tailed critic error of workload 3 is workload synthesis, not part of the method: the
     # scaled |delta| array that the priority stage reads is prepared once from the same td_delta the
@@ -253,6 +334,8 @@ def run_ours(args):
     distrl.distrl_retrace_targets(main_set.batch, w.gamma, w.lam, vt, adv, dl, main_set.lp_out, main_set.lm_out,
                                   workspace=ws_r)
     prio_in = (dl * tail) if tail is not None else dl
+    # real masses before the rounds are recorded below (their first, unrecorded run draws from q)
+    distrl.distrl_compute_priorities(prio_in, main_set.lp_buf, main_set.lm_buf, main_set.dv["entropy"], cfg, None, q)
     torch.cuda.synchronize()
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
@@ -286,7 +369,8 @@ def run_ours(args):
             rounds(s_graph, ins)
         torch.cuda.synchronize()
 
-    record_rounds(main_set)
+    for ins_ in sets:
+        record_rounds(ins_)
 
     def step(marks=None, ins=main_set):
         if args.fused:   # Retrace + priorities + sampler build in one pass over the buffer
@@ -323,8 +407,8 @@ def run_ours(args):
 
     uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", "")
     clocks = ClockSampler(uuid)
-    for _ in range(max(args.warmup, 3)):
-        step()
+    for i in range(max(args.warmup, 3)):
+        step(ins=sets[i & 1])
     barrier()
     marks = [[ev() for _ in range(5)] for _ in range(args.steps)]
     t_begin, t_end = ev(), ev()
@@ -332,12 +416,13 @@ def run_ours(args):
     clocks.mark()
     t_begin.record()
     for i in range(args.steps):
-        step(marks[i])
+        step(marks[i], ins=sets[i & 1])
     t_end.record()
     barrier()
     clk = clocks.stop()
     total_ms = t_begin.elapsed_time(t_end)
-    stage_ms = np.array([[m[i].elapsed_time(m[i + 1]) for i in range(4)] for m in marks]).mean(axis=0)
+    stage_all = np.array([[m[i].elapsed_time(m[i + 1]) for i in range(4)] for m in marks])
+    stage_ms, stage_med, stage_min = stage_all.mean(axis=0), np.median(stage_all, axis=0), stage_all.min(axis=0)
     st_r = distrl.distrl_get_status(ws_r)
     st_s = distrl.distrl_get_status(ws_s)
     if st_r or st_s:
@@ -356,8 +441,6 @@ def run_ours(args):
     e2e_steps = max(4, min(args.steps, 8))
     e2e_ms = float("nan")
     if not args.no_e2e:
-        sets = [main_set, InputSet()]
-        record_rounds(sets[1])
         main_stream = torch.cuda.current_stream()
         up_stream, down_stream = torch.cuda.Stream(), torch.cuda.Stream()
         plain = lambda: torch.cuda.Event()
@@ -462,21 +545,13 @@ def run_ours(args):
         return 0
 
     peak, peak_kind = _peaks()
-    if tok:   # r, V, step offsets, both bf16 token arrays in; v_target, advantage, td_delta, logpi, logmu out; offsets
-        retrace_bytes = (8 + 8 + 20) * n + 4 * int(a["step_token_offsets"][-1]) + 8 * (w.m + 1)
-    else:     # r, V, logpi, logmu in; v_target, advantage, td_delta out; offsets
-        retrace_bytes = 28 * n + 8 * (w.m + 1)
-    prio_bytes = 20 * n                          # delta, logpi, logmu, entropy in; q out
-    build_bytes = 4 * n + 8 * (n // 128)
-    if args.fused:   # r, V, logpi, logmu, entropy (+ scale) in; v_target, advantage, q out; offsets; tree levels 1-2
-        retrace_bytes = (20 + (4 if tail is not None else 0) + 12) * n + 8 * (w.m + 1) + 8 * (n // 128)
+    retrace_bytes, prio_bytes, build_bytes = _step_bytes(w, args)
     ach = retrace_bytes / (stage_ms[0] * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": world * n / (ms_per_step * 1e-3), "unit": METRIC, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": _config(w, args, l2="inputs larger than L2 (%.0f MB touched per step)" %
-                          ((retrace_bytes + prio_bytes + build_bytes) / 1e6)),
+        "config": _config(w, args),
         "stages": {
             # with --fused the first stage is the one fused pass and the next two are empty
             "retrace_ms": float(stage_ms[0]), "priorities_ms": None if args.fused else float(stage_ms[1]),
@@ -486,14 +561,20 @@ def run_ours(args):
             "samples_per_s": R * k / (stage_ms[3] * 1e-3),
             "priorities_gbs": None if args.fused else prio_bytes / (stage_ms[1] * 1e-3) / 1e9,
             "build_sampler_gbs": None if args.fused else build_bytes / (stage_ms[2] * 1e-3) / 1e9,
+            # the figures above are means over the timed steps; median and minimum of the same per-step timings
+            "median_ms": {"retrace": float(stage_med[0]), "priorities": None if args.fused else float(stage_med[1]),
+                          "build_sampler": None if args.fused else float(stage_med[2]), "rounds": float(stage_med[3])},
+            "min_ms": {"retrace": float(stage_min[0]), "priorities": None if args.fused else float(stage_min[1]),
+                       "build_sampler": None if args.fused else float(stage_min[2]), "rounds": float(stage_min[3])},
+            "timed_steps": int(args.steps),
         },
         "roofline": {"bound": "hbm", "kernel": ("scan_mask_kernel + scan_pipe_kernel<fused> (distrl_retrace_priorities_build)" if args.fused else "scan_mask_kernel + %s (distrl_retrace_targets)" % ("scan_tok_pipe_kernel (+ two stand-ins that return at once)" if tok else "scan_pipe_kernel")), "achieved": ach, "peak": peak,
                      "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
-                     "frac_of_nominal_8000": ach / 8000.0, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name) if (args.n_override is None and not args.fused) else None,
+                     "frac_of_nominal_8000": ach / 8000.0, "traffic": _measured_traffic(w.name) if (args.n_override is None and not args.fused) else None,
                      "algorithmic_bytes": retrace_bytes},
         "e2e": {"value": world * n / (e2e_ms * 1e-3) if e2e_ms == e2e_ms else None, "unit": METRIC,
                 "ms_per_step": e2e_ms if e2e_ms == e2e_ms else None,   # None: leg skipped with --no-e2e
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clk,
     }
@@ -501,22 +582,34 @@ def run_ours(args):
         line["next_rows"] = next_rows
     if not args.no_cpu_baseline and world == 1:
         est, desc, _ = _oracle_sample(w, 2_000_000, draws=48)
-        line["cpu_baseline"] = {"value": w.n / est, "unit": METRIC, "cores": 1, "kind": "oracle", "sample": desc}
+        line["cpu_baseline"] = {"value": w.n / est, "unit": METRIC, "cores": 1, "kind": "oracle", "sample": desc,
+                                "estimated": True}
+        if not tok:
+            try:
+                v_mc, cores, desc_mc = _oracle_all_cores(w)
+                line["cpu_baseline"]["multi_core"] = {"value": v_mc, "unit": "transitions/s (Retrace + priority only)",
+                                                      "cores": cores, "kind": "oracle", "sample": desc_mc}
+            except Exception as e:   # the one-core figure stands on its own
+                line["cpu_baseline"]["multi_core"] = {"value": None, "error": repr(e)[:200]}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
     return 0
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the Retrace call's kernels, from the ncu captures
-# summarised under profiles/:
-#   "large": scan_pipe_kernel 270.60 + 152.89 MB and scan_mask_kernel 11.28 MB, captured at full size
-#            (profiles/scan_pipe_kernel_large.md);
-#   "token": scan_tok_pipe_kernel 344.49 + 64.17 MB, scan_mask_kernel 2.19 MB and the two stand-ins that return at
-#            once 0.06 MB on a 4,194,304-step case of the same workload, scaled by 16 to the full 67,108,864 steps
-#            (every array grows in proportion) (profiles/scan_tok_pipe_kernel_token.md).
-# Other workloads have no capture: reported as null.
-TRAFFIC_BYTES_PER_LAUNCH = {"large": 434_770_000, "token": 16 * 410_910_000}
+def _measured_traffic(workload_name):
+    """dram__bytes_read.sum + dram__bytes_write.sum per call of the Retrace entry point, from the profiler capture
+    recorded in profiles/traffic.json (written by `python -m paper_2410_14803_b200.ncu_summary`).  The record names
+    the kernel sources it was taken with; once they have changed the counters are stale and None is reported."""
+    try:
+        from paper_2410_14803_b200 import ncu_summary
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            rec = json.load(f).get(workload_name)
+        if not rec or rec.get("source_sha256") != ncu_summary.kernel_sources_sha256():
+            return None
+        return int(rec["bytes_per_call"])
+    except Exception:
+        return None
 
 
 def main():
