@@ -605,7 +605,7 @@ def _measured_traffic(workload_name):
         from paper_2410_14803_b200 import ncu_summary
         with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
             rec = json.load(f).get(workload_name)
-        if not rec or rec.get("source_sha256") != ncu_summary.kernel_sources_sha256():
+        if not rec or rec.get("source_sha256") != ncu_summary.kernel_sources_sha256(rec.get("sources")):
             return None
         return int(rec["bytes_per_call"])
     except Exception:

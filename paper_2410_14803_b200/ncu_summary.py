@@ -45,11 +45,11 @@ COUNTERS = ["gpu__time_duration.sum", "dram__bytes_read.sum", "dram__bytes_write
             "sm__inst_issued.avg.pct_of_peak_sustained_active"]
 
 
-def kernel_sources_sha256() -> str:
-    """Hash of every kernel source file of the library, in name order."""
+def kernel_sources_sha256(names=None) -> str:
+    """Hash of the named kernel source files under csrc/ (default: all of them), in name order."""
     h = hashlib.sha256()
     d = os.path.join(_PKG, "csrc")
-    for name in sorted(os.listdir(d)):
+    for name in sorted(names if names else os.listdir(d)):
         if name.endswith((".cu", ".cuh")):
             h.update(name.encode())
             with open(os.path.join(d, name), "rb") as f:
@@ -128,7 +128,7 @@ def counters_table(path) -> str:
     return "\n".join(lines)
 
 
-def traffic_record(path, kernels: str, scale: float):
+def traffic_record(path, kernels: str, scale: float, sources):
     pat = re.compile(kernels)
     per = OrderedDict()
     for k, vals in read_raw(path):
@@ -140,7 +140,7 @@ def traffic_record(path, kernels: str, scale: float):
     return {"bytes_per_call": int(round(sum(kern.values()))),
             "kernels": {k: int(round(v)) for k, v in kern.items()},
             "launches_captured": {k: len(v) for k, v in per.items()},
-            "scaled_by": scale, "source_sha256": kernel_sources_sha256()}
+            "scaled_by": scale, "sources": sorted(sources), "source_sha256": kernel_sources_sha256(sources)}
 
 
 def main(argv=None):
@@ -155,6 +155,8 @@ def main(argv=None):
     a.add_argument("--workload", required=True)
     a.add_argument("--kernels", required=True, help="regular expression over the short kernel names of one call")
     a.add_argument("--scale", type=float, default=1.0, help="units of a full launch / units of the captured one")
+    a.add_argument("--sources", default="retrace.cu,common.cuh,priority.cuh,sampler.cuh",
+                   help="files under csrc/ that the captured kernels are compiled from")
     a.add_argument("--command", default="", help="the capture command, kept in the record")
     a.add_argument("--note", default="")
     args = ap.parse_args(argv)
@@ -163,7 +165,7 @@ def main(argv=None):
     elif args.what == "counters":
         print(counters_table(args.csv))
     else:
-        rec = traffic_record(args.csv, args.kernels, args.scale)
+        rec = traffic_record(args.csv, args.kernels, args.scale, [x for x in args.sources.split(",") if x])
         rec["command"] = args.command
         if args.note:
             rec["note"] = args.note
