@@ -69,13 +69,17 @@ static inline int one_wave_blocks(K kernel, int threads, size_t smem = 0) {
 struct WorkspaceHeader {
     int status;          // sticky device-side status word (distrl_status)
     unsigned int ticket; // dynamic tile counter of the scan
-    unsigned int qmin;   // batch minimum of sampled masses (sampler)
-    unsigned int done;   // finished-block counter (sampler)
+    unsigned int qmin;   // (unused)
+    unsigned int done;   // finished-block counter (sampler, draws normalised by the last block)
     unsigned int bad_epoch; // call number whose offsets failed validation (scan)
-    unsigned int left;      // blocks that have taken the batch minimum and are leaving (sampler)
+    unsigned int left;      // (unused)
     unsigned int tok_dense; // token-level scan: the steps own too many tokens on average for the pipelined kernel
     unsigned int pad_;
     unsigned long long scan_ticket; // pipelined fp32 scan: (number of the call << 32) | tiles handed out so far
+    // sampler, draws whose blocks wait for one another: two words (low half: batch minimum of the sampled
+    // masses, high half: blocks counted in) that take turns, and which of them the next call uses
+    unsigned long long pair[2];
+    unsigned int phase;
 };
 static_assert(sizeof(WorkspaceHeader) <= 256, "the header has 256 bytes");
 constexpr size_t kHeaderBytes = 256;

@@ -10,10 +10,12 @@
 //            finishes the levels above;
 //   sample : one warp per draw; per level one coalesced 256-byte load, a
 //            shuffle prefix sum and a ballot; the top levels sit in shared memory;
-//   update : a claim word per transition elects, for every distinct index, the
-//            highest batch position (what a sequential loop would leave); the
-//            winners store the new mass and add new - old to every ancestor, so
-//            the tree stays bit-identical to a rebuild.
+//   update : for every distinct index the highest batch position wins (what a
+//            sequential loop would leave) -- elected per block through a small
+//            hash table in shared memory for batches of up to 8192 positions,
+//            through a claim word per transition beyond that; the winners store
+//            the new mass and add new - old to every ancestor, so the tree stays
+//            bit-identical to a rebuild.
 #include "priority.cuh"
 #include "sampler.cuh"
 
@@ -108,11 +110,7 @@ __global__ void __launch_bounds__(256) build_leaf_kernel(Tree t, int vec_ok) {
     __shared__ unsigned long long s_l1[kFan];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     grid_launch_dependents(); // pass 2 may be scheduled now; it waits for this grid before it reads
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        t.hdr->qmin = 0xffffffffu;
-        t.hdr->done = 0u;
-        t.hdr->left = 0u;
-    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) sampler_handshake_reset(t.hdr);
     const int64_t g0 = (int64_t)blockIdx.x * kFan + warp * 4;
     unsigned long long s[4];
     if (vec_ok && (g0 + 4) * kLeaf <= t.n) {
@@ -177,6 +175,12 @@ __global__ void total_kernel(Tree t, unsigned long long *out) {
 // shared memory once per block, so a draw pays one global round trip for that
 // copy plus one per remaining level and one for the leaf group.
 // ---------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long *p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ int pick_lane(unsigned long long incl, unsigned long long v, unsigned long long y) {
     unsigned int mask = __ballot_sync(0xffffffffu, incl > y);
     if (mask) return __ffs(mask) - 1;
@@ -217,6 +221,8 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     }
     const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const unsigned long long uj = (j < k) ? __ldg(u + j) : 0ull; // in flight while the cache fills
+    // which of the two hand-shake words this call uses (it is flipped only after every block has counted itself in)
+    const unsigned int phase = (together && threadIdx.x == 0) ? (__ldcg(&t.hdr->phase) & 1u) : 0u;
     __syncthreads(); // the barrier object is initialised
     {
         unsigned int spins = 0;
@@ -275,9 +281,11 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
         y -= __shfl_sync(0xffffffffu, incl - v, c);
         if (lane == c) {
             int e = 0;
-            while (e < 3 && y >= qv[e]) { y -= qv[e]; ++e; }
+#pragma unroll
+            for (int f = 0; f < 3; ++f)
+                if (e == f && y >= qv[f]) { y -= qv[f]; e = f + 1; }
             int64_t idx = p + e;
-            uint32_t qs = qv[e];
+            uint32_t qs = (e == 0) ? qv[0] : (e == 1) ? qv[1] : (e == 2) ? qv[2] : qv[3];
             if (idx >= t.n) { idx = t.n - 1; qs = 1u; set_status(&t.hdr->status, DISTRL_ERR_INDEX); }
             idx_out[j] = idx;
             if (w_out) {
@@ -295,35 +303,35 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
     }
     if (!(w_out && normalise)) return;
     if (together) {
-        // Every block of the grid is resident at once (the host checked that the grid fits), so the
-        // blocks can wait for one another: each adds its smallest mass to the batch minimum, counts
-        // itself in and polls the count; when it is complete the minimum is final and every draw is
-        // rescaled from its register.  The largest weight belongs to the smallest sampled mass, so
-        // w_j = (q_j / q_min)^-beta.  The wait is bounded; the last block to leave resets the words.
+        // Every block of the grid is resident at once (cooperative launch), so the blocks can wait for one
+        // another.  Each adds its smallest mass to a batch minimum and counts itself in; minimum and count are
+        // the two halves of one 8-byte word, so a single load tells a waiting block both that everybody has
+        // arrived and what the minimum is.  Two such words take turns: the block that arrives last clears the
+        // other one and flips the phase for the next call, so nobody has to come back and tidy up.  The
+        // largest weight belongs to the smallest sampled mass: w_j = (q_j / q_min)^-beta.  The wait is bounded.
         if (mine) atomicMin(&s_qmin, my_q);
         __syncthreads();
         if (threadIdx.x == 0) {
-            atomicMin(&t.hdr->qmin, s_qmin);
+            unsigned long long *pair = &t.hdr->pair[phase];
+            unsigned int *half = reinterpret_cast<unsigned int *>(pair); // [0]: minimum, [1]: blocks counted in
+            atomicMin(&half[0], s_qmin);
             unsigned int seen;
-            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(seen) : "l"(&t.hdr->done) : "memory");
-            ++seen;
-            unsigned int spins = 0;
-            while (seen < gridDim.x) {
-                if (++spins > (1u << 22)) { set_status(&t.hdr->status, DISTRL_ERR_TIMEOUT); break; }
-                seen = ld_acquire_u32(&t.hdr->done);
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(seen) : "l"(&half[1]) : "memory");
+            if (seen + 1u == gridDim.x) {
+                // the last to arrive: the other word was read for the last time one call ago
+                t.hdr->pair[phase ^ 1u] = 0xffffffffull; // minimum: none yet; count: 0
+                st_release_u32(&t.hdr->phase, phase ^ 1u);
             }
-            s_qmin = __ldcg(&t.hdr->qmin);
+            unsigned long long both = ld_acquire_u64(pair);
+            unsigned int spins = 0;
+            while ((unsigned int)(both >> 32) < gridDim.x) {
+                if (++spins > (1u << 22)) { set_status(&t.hdr->status, DISTRL_ERR_TIMEOUT); break; }
+                both = ld_acquire_u64(pair);
+            }
+            s_qmin = (unsigned int)both;
         }
         __syncthreads();
-        if (mine) w_out[j] = s_nothing ? 0.f : powf((float)((double)my_q / (double)s_qmin), -beta);
-        if (threadIdx.x == 0) {
-            const unsigned int gone = atomicAdd(&t.hdr->left, 1u);
-            if (gone == gridDim.x - 1) { // everybody has read the minimum: ready for the next call
-                t.hdr->qmin = 0xffffffffu;
-                t.hdr->done = 0u;
-                t.hdr->left = 0u;
-            }
-        }
+        if (mine) w_out[j] = s_nothing ? 0.f : powf((float)my_q / (float)s_qmin, -beta);
         return;
     }
     // The block that finishes last divides by the batch maximum.  The largest weight belongs to the
@@ -485,35 +493,55 @@ __global__ void __launch_bounds__(kUpdateThreads) update_apply_kernel(Tree t, Up
 
 // ---------------------------------------------------------------------------
 // update of a small batch in one launch.  For k <= kSmallBatch the election needs
-// no claim table and no second kernel: every block stages the batch's indices in
-// shared memory and a warp decides for its position j by looking at the positions
-// after it -- j applies its value iff no later position holds the same index,
-// which is what a sequential loop over the batch leaves.  The k^2 / 2 comparisons
-// (16-byte shared-memory loads, four indices each) cost less than a launch.
+// no claim table in global memory and no second kernel.  A sequential loop over
+// the batch leaves, for an index that occurs several times, the value of its
+// highest position; so position j applies its value iff no later position holds
+// the same index.  Every block answers that for its own 32 positions: it puts
+// their indices into a small hash table in shared memory, then all its threads
+// stream the whole batch past that table (one probe per batch entry, almost
+// always of an empty slot) and record, per table entry, the highest position at
+// which its index occurs.  O(k) work per block, the same for every block.
 // ---------------------------------------------------------------------------
 constexpr int kSmallBatch = 8192;       // positions the single-launch update serves
 constexpr int kSmallThreads = 512;
-constexpr int kSmallPerWarp = 2;        // batch positions per warp
+constexpr int kSmallPerWarp = 2;        // batch positions per warp (one was slower in a chain of rounds, four much slower)
 constexpr int kSmallPerBlock = (kSmallThreads / 32) * kSmallPerWarp;
-constexpr unsigned int kNoIndex = 0xffffffffu; // staged in place of an index outside [0, n)
+constexpr int kSmallSlots = 4 * kSmallPerBlock;      // hash-table slots of a block (four per position it owns)
+constexpr int kSmallKeep = 8;           // batch entries a thread keeps in registers (covers k <= 4096)
+constexpr unsigned int kNoIndex = 0xffffffffu; // an empty slot; never a valid index (n < 2^31 on this path)
+
+__device__ __forceinline__ unsigned int slot_of(unsigned int i) { return ((i * 2654435761u) >> 16) & (kSmallSlots - 1); }
 
 __global__ void __launch_bounds__(kSmallThreads) update_small_kernel(
     Tree t, const int64_t *__restrict__ idx, int k, const float *__restrict__ new_abs_delta,
     const float *__restrict__ lp, const float *__restrict__ lm, const float *__restrict__ ent, PrioCfg c,
     float *__restrict__ mass_out) {
-    __shared__ __align__(16) unsigned int s_idx[kSmallBatch]; // low words of the batch's indices (n < 2^31 here)
+    __shared__ unsigned int s_key[kSmallSlots]; // low words of the indices of this block's positions
+    __shared__ int s_last[kSmallSlots];         // highest batch position that holds the slot's index
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < kSmallSlots; i += kSmallThreads) { s_key[i] = kNoIndex; s_last[i] = -1; }
     grid_dependency_wait();
     grid_launch_dependents();
-    // this block's positions first: their gathers are in flight while the batch is staged
+    // Every load that depends on nothing goes out first: this warp's own indices, then the thread's share of
+    // the whole batch.  The gathers follow as soon as the own indices are there.
     const int j0 = blockIdx.x * kSmallPerBlock + warp * kSmallPerWarp;
     int64_t my_i[kSmallPerWarp];
+#pragma unroll
+    for (int u = 0; u < kSmallPerWarp; ++u) my_i[u] = (j0 + u < k) ? idx[j0 + u] : -1;
+    int64_t kept[kSmallKeep];
+#pragma unroll
+    for (int e = 0; e < kSmallKeep; ++e) {
+        const int p = threadIdx.x + e * kSmallThreads;
+        kept[e] = (p < k) ? idx[p] : -1;
+    }
+    __syncthreads(); // the table is empty
     float g_val[kSmallPerWarp]; // lane 0: log pi, lane 1: log mu, lane 2: entropy, lane 3: old mass (bits), lane 4: |delta|
+    int my_slot[kSmallPerWarp];
 #pragma unroll
     for (int u = 0; u < kSmallPerWarp; ++u) {
         const int j = j0 + u;
-        my_i[u] = (j < k) ? idx[j] : -1;
         g_val[u] = 0.f;
+        my_slot[u] = -1;
         if (my_i[u] >= 0 && my_i[u] < t.n) {
             const int64_t i = my_i[u];
             if (lane == 0) g_val[u] = __ldg(lp + i);
@@ -521,14 +549,36 @@ __global__ void __launch_bounds__(kSmallThreads) update_small_kernel(
             else if (lane == 2) g_val[u] = ent ? __ldg(ent + i) : 0.f;
             else if (lane == 3) g_val[u] = __uint_as_float(__ldcg(t.q + i));
             else if (lane == 4) g_val[u] = new_abs_delta[j];
+            if (lane == 0) { // claim a slot for this index (another position of the block may hold the same one)
+                const unsigned int key = (unsigned int)i;
+                unsigned int h = slot_of(key);
+                for (int probe = 0; probe < kSmallSlots; ++probe) { // the table is a quarter full at most: ends early
+                    const unsigned int was = atomicCAS(&s_key[h], kNoIndex, key);
+                    if (was == kNoIndex || was == key) { my_slot[u] = (int)h; break; }
+                    h = (h + 1) & (kSmallSlots - 1);
+                }
+            }
         }
     }
-    const int kpad = (k + 3) & ~3;
-    for (int p = threadIdx.x; p < kpad; p += kSmallThreads) {
-        const int64_t i = (p < k) ? idx[p] : -1;
-        s_idx[p] = (i >= 0 && i < t.n) ? (unsigned int)i : kNoIndex;
-    }
-    __syncthreads();
+    // (the batch entries were sent for before the table was set up: keep them from being fetched only now)
+#pragma unroll
+    for (int e = 0; e < kSmallKeep; ++e) asm volatile("" : "+l"(kept[e]));
+    __syncthreads(); // the table holds this block's indices
+    auto note = [&](int p, int64_t i) { // batch position p holds index i: is it one of ours?
+        if (i < 0 || i >= t.n) return;
+        const unsigned int key = (unsigned int)i;
+        unsigned int h = slot_of(key);
+        for (int probe = 0; probe < kSmallSlots; ++probe) {
+            const unsigned int at = s_key[h];
+            if (at == kNoIndex) return;
+            if (at == key) { atomicMax(&s_last[h], p); return; }
+            h = (h + 1) & (kSmallSlots - 1);
+        }
+    };
+#pragma unroll
+    for (int e = 0; e < kSmallKeep; ++e) note(threadIdx.x + e * kSmallThreads, kept[e]);
+    for (int p = threadIdx.x + kSmallKeep * kSmallThreads; p < k; p += kSmallThreads) note(p, idx[p]);
+    __syncthreads(); // every occurrence has been recorded
 #pragma unroll
     for (int u = 0; u < kSmallPerWarp; ++u) {
         const int j = j0 + u;
@@ -541,25 +591,22 @@ __global__ void __launch_bounds__(kSmallThreads) update_small_kernel(
             }
             continue;
         }
-        // does a later position hold the same index?
-        const unsigned int key = (unsigned int)i;
-        bool later = false;
-        for (int b = ((j + 1) & ~3) + 4 * lane; b < kpad; b += 128) {
-            const uint4 v = *reinterpret_cast<const uint4 *>(&s_idx[b]);
-            later |= (b > j && v.x == key) | (b + 1 > j && v.y == key) | (b + 2 > j && v.z == key) | (b + 3 > j && v.w == key);
-        }
-        later = __any_sync(0xffffffffu, later);
         const float p = __shfl_sync(0xffffffffu, g_val[u], 0), m = __shfl_sync(0xffffffffu, g_val[u], 1);
         const float h_in = __shfl_sync(0xffffffffu, g_val[u], 2);
         const uint32_t qo = __float_as_uint(__shfl_sync(0xffffffffu, g_val[u], 3));
         const float nd = __shfl_sync(0xffffffffu, g_val[u], 4);
         if (lane == 0) {
+            const bool later = my_slot[u] >= 0 && s_last[my_slot[u]] > j; // a later position holds the same index
             const float mass = prio_mass(nd, p, m, ent ? h_in : -p, c);
             if (mass_out) mass_out[j] = mass;
             const uint32_t qn = prio_quantise(mass, c);
             if (!later && qn != qo) {
                 t.q[i] = qn;
                 const unsigned long long diff = (unsigned long long)qn - (unsigned long long)qo; // mod 2^64
+                // Plain reductions on every level, the few top entries included: summing those per block in
+                // shared memory and flushing after a barrier was measured again (per-kernel +1.1 us, no gain
+                // for a round), although the top entries' additions, a quarter of the batch each, do delay the
+                // draw that follows by about 1 us.
                 int64_t node = i / kLeaf;
                 for (int l = 1; l <= t.levels; ++l) {
                     atomicAdd(&t.lvl[l][node], diff); // result unused: a reduction the thread does not wait for

@@ -15,6 +15,17 @@ struct TreeBase {
     WorkspaceHeader *hdr;
 };
 
+// The words through which the blocks of a normalising draw wait for one another, as a freshly built
+// sampler has them (device side; called by whichever kernel builds the tree).
+#ifdef __CUDACC__
+__device__ __forceinline__ void sampler_handshake_reset(WorkspaceHeader *hdr) {
+    hdr->done = 0u;
+    hdr->pair[0] = 0xffffffffull; // minimum: none yet; count: 0
+    hdr->pair[1] = 0xffffffffull;
+    hdr->phase = 0u;
+}
+#endif
+
 // Validates the arguments and fills a host handle over `workspace`; launches nothing.
 int sampler_create(uint32_t *prio_q, int64_t n, void *workspace, size_t workspace_bytes, distrl_sampler **out);
 void sampler_tree_base(const distrl_sampler *s, TreeBase *out);
