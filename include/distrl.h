@@ -128,10 +128,18 @@ int distrl_retrace_targets(const distrl_batch *batch, float gamma, float lambda,
  *   status_out_device : device int or NULL; receives the device status word of
  *       this call (DISTRL_OK, DISTRL_ERR_OFFSETS, DISTRL_ERR_TIMEOUT).
  * The call allocates nothing (no cudaMalloc / cudaFree, no library allocator).
- * The first call on each device looks up the array's device address; make that
- * first call outside any stream capture.  All calls on a device share the one
- * array: issue them on one stream, or otherwise make sure two of them never
- * run on the GPU at the same time -- overlapping calls race on it.
+ * One thing happens once per device all the same: the first call looks up the
+ * array's device address, and, if nothing of this library has run on the device
+ * yet, the CUDA runtime loads the library's code and the array at that moment
+ * (device memory the runtime takes, about 1 MB).  So make one warm-up call per
+ * device early -- before a framework reserves what is left of the GPU, and
+ * outside any stream capture -- and later calls touch no allocator at all.
+ * Arguments are checked before anything is enqueued: a refused call leaves the
+ * array as it was.  All calls on a device share the one array: issue them on one
+ * stream, or otherwise make sure two of them never run on the GPU at the same
+ * time -- overlapping calls race on it.  (Calls of distrl_retrace_targets with
+ * their own workspaces are not affected and may run beside it.)  First calls
+ * from several host threads at once are safe.
  */
 #define DISTRL_STATIC_MAX_N ((int64_t)1 << 22)
 int distrl_retrace_targets_static(const distrl_batch *batch, float gamma, float lambda,
@@ -434,6 +442,17 @@ int distrl_selftest_bounded_wait(void *workspace, size_t workspace_bytes, void *
  * block only ever waits for tiles of blocks that are already running.)
  */
 int distrl_set_cooperative_launch(int allowed);
+
+/*
+ * Checked build (no counterpart in the paper).  A library compiled with
+ * -DDISTRL_BOUNDS_CHECK range-checks every index its kernels compute right before
+ * the access; an index out of range is recorded and the access skipped (nothing
+ * traps, nothing is touched out of bounds).  Returns 1 if this library is such a
+ * build, else 0 (record all zero).  Synchronises the device, copies
+ * {violations, source line of the first, its index, its limit} to record4_host
+ * (host int64[4]) and clears the record.  The ordinary build carries no checks.
+ */
+int distrl_bounds_report(int64_t *record4_host);
 
 const char *distrl_error_string(int code);
 const char *distrl_last_cuda_error(void); /* text of the last failed CUDA call, this thread */

@@ -63,6 +63,42 @@ def _load():
     path = _build.LIB_PATH
     if not os.path.exists(path):
         path = _build.build()
+    _lib = _open(path)
+    return _lib
+
+
+_checked_lib = None
+
+
+class checked_build:
+    """Context manager: inside it every call of this module goes to the range-checked build of the library
+    (compiled on first use).  On exit the ordinary library is back and `violations` holds what the checks
+    recorded: (count, source line of the first, its index, its limit)."""
+
+    def __enter__(self):
+        global _lib, _checked_lib
+        if _checked_lib is None:
+            _checked_lib = _open(_build.build(checked=True))
+        self._saved = _load()
+        _lib = _checked_lib
+        self.report()          # start from a clean record
+        return self
+
+    def report(self):
+        rec = (ctypes.c_int64 * 4)()
+        rc = _checked_lib.distrl_bounds_report(rec)
+        if rc != 1:
+            raise DistrlError(rc, "distrl_bounds_report (not a checked build?)")
+        return tuple(int(x) for x in rec)
+
+    def __exit__(self, *exc):
+        global _lib
+        self.violations = self.report()
+        _lib = self._saved
+        return False
+
+
+def _open(path):
     lib = ctypes.CDLL(path)
     vp, i64, sz, f32, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_float, ctypes.c_int
     sig = {
@@ -96,6 +132,7 @@ def _load():
         "distrl_get_status": (ci, [vp, vp]),
         "distrl_selftest_bounded_wait": (ci, [vp, sz, vp]),
         "distrl_set_cooperative_launch": (ci, [ci]),
+        "distrl_bounds_report": (ci, [vp]),
         "distrl_error_string": (ctypes.c_char_p, [ci]),
         "distrl_last_cuda_error": (ctypes.c_char_p, []),
         "distrl_version": (ctypes.c_char_p, []),
@@ -103,7 +140,6 @@ def _load():
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
         fn.restype, fn.argtypes = res, args
-    _lib = lib
     return lib
 
 

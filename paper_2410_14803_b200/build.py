@@ -10,6 +10,10 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libdistrl_b200.so")
+# The checked build: every computed index is range-checked (DISTRL_BOUNDS_CHECK) and the pipelined scan runs
+# with tiles of half the size (4 items per thread), so the same inputs are cut into tiles differently.
+CHECKED_LIB_PATH = os.path.join(_PKG, "libdistrl_b200_checked.so")
+CHECKED_FLAGS = ["-DDISTRL_BOUNDS_CHECK", "-DDISTRL_PIPE_ITEMS=4"]
 SOURCES = ["api.cu", "retrace.cu", "priority.cu", "sampler.cu", "batch.cu", "replay.cu"]
 
 
@@ -19,22 +23,23 @@ def _newest_source_mtime() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into libdistrl_b200.so (no GPU needed)."""
-    if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= _newest_source_mtime():
-        return LIB_PATH
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compile every .cu under csrc/ into libdistrl_b200.so (no GPU needed); checked=True: the checked build."""
+    out = CHECKED_LIB_PATH if checked else LIB_PATH
+    if not force and os.path.exists(out) and os.path.getmtime(out) >= _newest_source_mtime():
+        return out
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB_PATH + ".tmp.%d" % os.getpid()
+    tmp = out + ".tmp.%d" % os.getpid()
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-t", "0", "-I", INCLUDE, "-I", CSRC, "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("DISTRL_NVCC_EXTRA", "").split()   # e.g. -D overrides of tuning constants
+    cmd += CHECKED_FLAGS if checked else os.environ.get("DISTRL_NVCC_EXTRA", "").split()   # e.g. -D overrides of tuning constants
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

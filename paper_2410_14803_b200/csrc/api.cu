@@ -9,6 +9,14 @@ namespace distrl {
 static std::atomic<int> g_cooperative{1};
 bool cooperative_launch_allowed() { return g_cooperative.load(std::memory_order_relaxed) != 0; }
 
+#ifdef DISTRL_BOUNDS_CHECK
+int bounds_take_retrace(long long *rec);
+int bounds_take_priority(long long *rec);
+int bounds_take_sampler(long long *rec);
+int bounds_take_batch(long long *rec);
+int bounds_take_replay(long long *rec);
+#endif
+
 static thread_local char g_cuda_error[256] = "";
 
 int record_cuda_error(cudaError_t e, const char *what) {
@@ -59,6 +67,25 @@ extern "C" const char *distrl_error_string(int code) {
 
 extern "C" int distrl_set_cooperative_launch(int allowed) {
     return g_cooperative.exchange(allowed ? 1 : 0, std::memory_order_relaxed);
+}
+
+extern "C" int distrl_bounds_report(int64_t *record4_host) {
+    if (!record4_host) return DISTRL_ERR_NULL;
+    for (int i = 0; i < 4; ++i) record4_host[i] = 0;
+#ifdef DISTRL_BOUNDS_CHECK
+    DISTRL_CUDA_TRY(cudaDeviceSynchronize());
+    int (*units[])(long long *) = {bounds_take_retrace, bounds_take_priority, bounds_take_sampler, bounds_take_batch,
+                                   bounds_take_replay};
+    for (auto take : units) {
+        long long rec[4] = {0, 0, 0, 0};
+        if (take(rec) != 0) return record_cuda_error(cudaGetLastError(), "distrl_bounds_report");
+        if (rec[0] && !record4_host[0]) { record4_host[1] = rec[1]; record4_host[2] = rec[2]; record4_host[3] = rec[3]; }
+        record4_host[0] += rec[0];
+    }
+    return 1;
+#else
+    return 0;
+#endif
 }
 
 extern "C" const char *distrl_last_cuda_error(void) { return g_cuda_error; }

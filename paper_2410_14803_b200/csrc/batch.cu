@@ -73,6 +73,7 @@ __global__ void __launch_bounds__(kBatchThreads) traj_ranges_kernel(
             end[j] = -1;
             continue;
         }
+        if (!DISTRL_IN(t + 1, m + 1)) continue;
         begin[j] = off[t];
         end[j] = off[t + 1];
     }
@@ -120,12 +121,12 @@ __global__ void __launch_bounds__(kBatchThreads) filter_kernel(
                     const int first = (wd == (lo >> 5)) ? (lo & 31) : 0;
                     const int last = (wd == ((hi - 1) >> 5)) ? ((hi - 1) & 31) : 31; // inclusive
                     const unsigned int bits = (0xFFFFFFFFu >> (31 - last)) & (0xFFFFFFFFu << first);
-                    atomicOr(&s_drop[wd], bits);
+                    if (DISTRL_IN(wd, kFilterWords)) atomicOr(&s_drop[wd], bits);
                 }
             }
             __syncthreads();
             for (int i = tid; i < cnt; i += kBatchThreads)
-                if ((s_drop[i >> 5] >> (i & 31)) & 1u) q[p + i] = 0u;
+                if (((s_drop[i >> 5] >> (i & 31)) & 1u) && DISTRL_IN(p + i, n)) q[p + i] = 0u;
             __syncthreads(); // the bitmap is cleared for the next window
         }
     }
@@ -208,3 +209,5 @@ extern "C" int distrl_filter_trajectories(int64_t n, int64_t m, const int64_t *t
     DISTRL_CUDA_TRY(cudaGetLastError());
     return DISTRL_OK;
 }
+
+DISTRL_BOUNDS_UNIT(batch, 4)

@@ -104,6 +104,52 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 // Records the first device-side error; later ones are dropped.
 __device__ __forceinline__ void set_status(int *status, int code) { atomicCAS(status, 0, code); }
 
+// Checked build (-DDISTRL_BOUNDS_CHECK): the stand-in for a memory checker.  Every index that a kernel
+// computes from its inputs or from its own tiling goes through DISTRL_IN(i, n) right before the access;
+// an index outside [0, n) is recorded (the first one: source line, index, limit; and a count of all) and
+// the access is skipped -- nothing traps and nothing is read or written out of bounds.  The record is
+// read with distrl_bounds_report().  In the ordinary build the macro is the constant true.
+#ifdef DISTRL_BOUNDS_CHECK
+// (one record per translation unit: the library is built without relocatable device code)
+static __device__ long long g_bounds_record[4]; // violations, line of the first one, its index, its limit
+static __device__ __noinline__ bool bounds_violation(long long i, long long n, int line) {
+    if (atomicAdd(reinterpret_cast<unsigned long long *>(&g_bounds_record[0]), 1ull) == 0ull) {
+        g_bounds_record[1] = line;
+        g_bounds_record[2] = i;
+        g_bounds_record[3] = n;
+    }
+    return false;
+}
+__device__ __forceinline__ bool bounds_ok(long long i, long long n, int line) {
+    return (i >= 0 && i < n) ? true : bounds_violation(i, n, line);
+}
+#define DISTRL_IN(i, n) (::distrl::bounds_ok((long long)(i), (long long)(n), __LINE__))
+#else
+#define DISTRL_IN(i, n) (true)
+#endif
+
+#endif // __CUDACC__
+
+// Each translation unit with kernels names itself once with DISTRL_BOUNDS_UNIT(name, id): in the checked build
+// that defines the function through which distrl_bounds_report() collects (and clears) the unit's record; the
+// line it reports is id * 100000 + source line.
+#if defined(__CUDACC__) && defined(DISTRL_BOUNDS_CHECK)
+#define DISTRL_BOUNDS_UNIT(name, id)                                                                   \
+    namespace distrl {                                                                                 \
+    int bounds_take_##name(long long *rec) {                                                           \
+        const long long zero[4] = {0, 0, 0, 0};                                                        \
+        if (cudaMemcpyFromSymbol(rec, g_bounds_record, sizeof(zero)) != cudaSuccess) return -1;        \
+        if (cudaMemcpyToSymbol(g_bounds_record, zero, sizeof(zero)) != cudaSuccess) return -1;         \
+        if (rec[0]) rec[1] += 100000LL * (id);                                                         \
+        return 0;                                                                                      \
+    }                                                                                                  \
+    }
+#else
+#define DISTRL_BOUNDS_UNIT(name, id)
+#endif
+
+#ifdef __CUDACC__
+
 // Streaming 128-bit loads/stores: data that is touched once should not evict
 // what the rest of the pass keeps in L2.
 __device__ __forceinline__ float4 ldg_stream_f4(const float *p) {

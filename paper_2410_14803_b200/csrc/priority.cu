@@ -222,3 +222,5 @@ extern "C" int distrl_compute_priorities_traj(int64_t n, int64_t m, const int64_
     DISTRL_CUDA_TRY(cudaGetLastError());
     return DISTRL_OK;
 }
+
+DISTRL_BOUNDS_UNIT(priority, 2)

@@ -75,13 +75,14 @@ struct FieldPtrs {
 __device__ __forceinline__ bool bit_at(const unsigned int *mask, int64_t i) { return (mask[i >> 5] >> (i & 31)) & 1u; }
 
 // bits [a, b) of `mask` set (value != 0) or cleared, word by word with one lane per word
-__device__ __forceinline__ void warp_fill_bits(unsigned int *mask, int64_t a, int64_t b, int value, int lane) {
+__device__ __forceinline__ void warp_fill_bits(unsigned int *mask, int64_t words, int64_t a, int64_t b, int value, int lane) {
     if (b <= a) return;
     for (int64_t w = (a >> 5) + lane; w <= ((b - 1) >> 5); w += 32) {
         const int64_t lo = w << 5;
         unsigned int m = 0xffffffffu;
         if (a > lo) m &= 0xffffffffu << (int)(a - lo);
         if (b < lo + 32) m &= 0xffffffffu >> (int)(lo + 32 - b);
+        if (!DISTRL_IN(w, words)) continue;
         if (value) atomicOr(&mask[w], m);
         else atomicAnd(&mask[w], ~m);
     }
@@ -121,7 +122,7 @@ __global__ void __launch_bounds__(32) ring_cut_kernel(RingWs ws, int64_t n, int6
         a = right;
         b = found < n ? found : n;
     }
-    warp_fill_bits(ws.alive, a, b, 0, lane);
+    warp_fill_bits(ws.alive, ws.words, a, b, 0, lane);
     if (lane == 0) {
         ws.hdr->kill[0] = a;
         ws.hdr->kill[1] = b;
@@ -145,8 +146,8 @@ __global__ void __launch_bounds__(kRingThreads) ring_cover_kernel(RingWs ws, Cov
         for (int64_t c = (r.a[i] >> 10) + warp; c <= ((r.b[i] - 1) >> 10); c += warps) {
             const int64_t lo = c << 10, hi = lo + 1024;
             const int64_t a = r.a[i] > lo ? r.a[i] : lo, b = r.b[i] < hi ? r.b[i] : hi;
-            warp_fill_bits(ws.start, a, b, 0, lane);
-            warp_fill_bits(ws.alive, a, b, r.alive[i], lane);
+            warp_fill_bits(ws.start, ws.words, a, b, 0, lane);
+            warp_fill_bits(ws.alive, ws.words, a, b, r.alive[i], lane);
         }
     }
 }
@@ -173,28 +174,30 @@ __global__ void __launch_bounds__(kRingThreads) ring_starts_kernel(RingWs ws, in
     }
     if (next == row) return; // an empty trajectory stores nothing
     const int64_t slot = row < split_row ? head + row : row - split_row;
-    if (slot >= 0 && slot < n) atomicOr(&ws.start[slot >> 5], 1u << (slot & 31));
+    if (slot >= 0 && slot < n && DISTRL_IN(slot >> 5, ws.words)) atomicOr(&ws.start[slot >> 5], 1u << (slot & 31));
 }
 
 // rows: new row t of every field goes to slot head + t (t < split_row) or t - split_row.
-__global__ void __launch_bounds__(kRingThreads) ring_rows_kernel(FieldPtrs f, int64_t total, int64_t head,
+__global__ void __launch_bounds__(kRingThreads) ring_rows_kernel(FieldPtrs f, int64_t n, int64_t total, int64_t head,
                                                                  int64_t split_row) {
     grid_dependency_wait();
     grid_launch_dependents();
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride) {
         const int64_t slot = t < split_row ? head + t : t - split_row;
+        if (!DISTRL_IN(slot, n)) continue;
         for (int i = 0; i < f.count; ++i) f.dst[i][slot] = __ldcs(f.src[i] + t);
     }
 }
 
 // masses without a sampler: plain stores (src null: zeros), and zeros for the killed range
-__global__ void __launch_bounds__(kRingThreads) ring_mass_run_kernel(uint32_t *__restrict__ q, int64_t a, int64_t b,
-                                                                     const uint32_t *__restrict__ src) {
+__global__ void __launch_bounds__(kRingThreads) ring_mass_run_kernel(uint32_t *__restrict__ q, int64_t n, int64_t a,
+                                                                     int64_t b, const uint32_t *__restrict__ src) {
     grid_dependency_wait();
     grid_launch_dependents();
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = a + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < b; i += stride) q[i] = src ? src[i - a] : 0u;
+    for (int64_t i = a + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < b; i += stride)
+        if (DISTRL_IN(i, n)) q[i] = src ? src[i - a] : 0u;
 }
 __global__ void __launch_bounds__(kRingThreads) ring_mass_kill_kernel(uint32_t *__restrict__ q, int64_t n,
                                                                       const long long *__restrict__ kill) {
@@ -463,7 +466,7 @@ extern "C" int distrl_replay_ingest(distrl_replay *rb, distrl_sampler *sampler, 
         for (int i = 0; i < rb->n_fields; ++i) { f.dst[i] = rb->field[i]; f.src[i] = new_fields[i]; }
         int64_t grid = ceil_div(total, kRingThreads);
         if (grid > 8 * 148) grid = 8 * 148;
-        DISTRL_CUDA_TRY(launch_pdl(ring_rows_kernel, dim3((unsigned)grid), dim3(kRingThreads), 0, st, f, total, head0,
+        DISTRL_CUDA_TRY(launch_pdl(ring_rows_kernel, dim3((unsigned)grid), dim3(kRingThreads), 0, st, f, n, total, head0,
                                    split_row));
     }
     // masses: the killed slots, the two runs of new rows, the retired stretch; one launch after the
@@ -479,7 +482,7 @@ extern "C" int distrl_replay_ingest(distrl_replay *rb, distrl_sampler *sampler, 
             if (b <= a) return cudaSuccess;
             int64_t grid = ceil_div(b - a, kRingThreads);
             if (grid > 8 * 148) grid = 8 * 148;
-            return launch_pdl(ring_mass_run_kernel, dim3((unsigned)grid), dim3(kRingThreads), 0, st, rb->q, a, b, src);
+            return launch_pdl(ring_mass_run_kernel, dim3((unsigned)grid), dim3(kRingThreads), 0, st, rb->q, n, a, b, src);
         };
         DISTRL_CUDA_TRY(launch_pdl(ring_mass_kill_kernel, dim3(1), dim3(kRingThreads), 0, st, rb->q, n,
                                    (const long long *)rb->ws.hdr->kill));
@@ -501,3 +504,5 @@ extern "C" int distrl_replay_destroy(distrl_replay *rb) {
     delete rb;
     return DISTRL_OK;
 }
+
+DISTRL_BOUNDS_UNIT(replay, 5)

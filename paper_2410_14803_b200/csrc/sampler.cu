@@ -239,7 +239,8 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
         // top level: its entries sum to the total mass
         int l = t.levels;
         unsigned long long v = 0ull;
-        if (lane < t.count[l]) v = (l >= tc.from) ? s_top[tc.off[l] + lane] : __ldcg(&t.lvl[l][lane]);
+        if (lane < t.count[l] && (l < tc.from || DISTRL_IN(tc.off[l] + lane, kTopCap)))
+            v = (l >= tc.from) ? s_top[tc.off[l] + lane] : __ldcg(&t.lvl[l][lane]);
         unsigned long long incl = warp_incl_scan_u64(v, lane);
         const unsigned long long total = __shfl_sync(0xffffffffu, incl, 31);
         unsigned long long y = __umul64hi(uj, total);
@@ -261,7 +262,8 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(
             node = node * kFan + c;
             if (--l == 0) break;
             int64_t i = node * kFan + lane;
-            if (i < t.count[l]) v = (l >= tc.from) ? s_top[tc.off[l] + (int)i] : __ldcg(&t.lvl[l][i]);
+            if (i < t.count[l] && (l < tc.from || DISTRL_IN(tc.off[l] + i, kTopCap)))
+                v = (l >= tc.from) ? s_top[tc.off[l] + (int)i] : __ldcg(&t.lvl[l][i]);
             else v = 0ull;
             incl = warp_incl_scan_u64(v, lane);
         }
@@ -476,6 +478,7 @@ __global__ void __launch_bounds__(kUpdateThreads) update_apply_kernel(Tree t, Up
                 const unsigned long long diff = (unsigned long long)qn - (unsigned long long)qo; // mod 2^64
                 int64_t node = i / kLeaf;
                 for (int l = 1; l <= t.levels; ++l) {
+                    if (!DISTRL_IN(node, t.count[l])) continue;
                     if (l >= acc_from) atomicAdd(&s_acc[s_acc_off[l] + (int)node], diff);
                     else atomicAdd(&t.lvl[l][node], diff);
                     node /= kFan;
@@ -609,7 +612,7 @@ __global__ void __launch_bounds__(kSmallThreads) update_small_kernel(
                 // draw that follows by about 1 us.
                 int64_t node = i / kLeaf;
                 for (int l = 1; l <= t.levels; ++l) {
-                    atomicAdd(&t.lvl[l][node], diff); // result unused: a reduction the thread does not wait for
+                    if (DISTRL_IN(node, t.count[l])) atomicAdd(&t.lvl[l][node], diff); // result unused: a reduction the thread does not wait for
                     node /= kFan;
                 }
             }
@@ -633,20 +636,20 @@ __device__ __forceinline__ void overwrite_group(const Tree &t, int64_t g, int64_
         const int64_t i = g * kLeaf + 4 * lane + e;
         uint32_t v = 0u;
         if (i < t.n) {
-            if (i >= a && i < b) { v = src ? src[i - a] : 0u; t.q[i] = v; }
+            if (i >= a && i < b && DISTRL_IN(i, t.n)) { v = src ? src[i - a] : 0u; t.q[i] = v; }
             else v = __ldcg(t.q + i);
         }
         sum += v;
     }
     sum = warp_sum_u64(sum);
-    if (lane == 0) {
+    if (lane == 0 && DISTRL_IN(g, t.count[1])) {
         const unsigned long long old = t.lvl[1][g];
         t.lvl[1][g] = sum; // this warp is the only writer of the group at this time
         const unsigned long long diff = sum - old; // mod 2^64
         if (diff) {
             int64_t node = g / kFan;
             for (int l = 2; l <= t.levels; ++l) {
-                atomicAdd(&t.lvl[l][node], diff);
+                if (DISTRL_IN(node, t.count[l])) atomicAdd(&t.lvl[l][node], diff);
                 node /= kFan;
             }
         }
@@ -912,3 +915,5 @@ extern "C" int distrl_destroy_sampler(distrl_sampler *s) {
     delete s;
     return DISTRL_OK;
 }
+
+DISTRL_BOUNDS_UNIT(sampler, 3)
