@@ -79,42 +79,57 @@ __global__ void __launch_bounds__(kBatchThreads) traj_ranges_kernel(
     }
 }
 
-// Trajectory filter: a block takes kBatchThreads consecutive trajectories, whose steps are one
-// contiguous range of the buffer, and walks that range in windows of kFilterWindow steps.  Per
-// window the thread of every trajectory that is not retained sets the bits of its steps in a
-// shared-memory bitmap (whole words at a time), then all threads sweep the window with coalesced
-// stores of zero where a bit is set.  Masses of retained trajectories are neither read nor written.
-constexpr int kFilterWindow = 4096;
+// Trajectory filter: a warp takes 32 consecutive trajectories, whose steps are one contiguous range of
+// the buffer, and walks that range in windows of kFilterWindow steps.  Per window the lane of every
+// trajectory that is not retained sets the bits of its steps in the warp's own bitmap in shared memory
+// (whole words at a time), then the warp sweeps the window, 32 consecutive steps per instruction, with
+// coalesced stores of zero where a bit is set.  Masses of retained trajectories are neither read nor
+// written.  Warps never meet at a block barrier; the loads of the next group of trajectories are sent
+// for before the current one is swept.
+constexpr int kFilterWindow = 2048;
 constexpr int kFilterWords = kFilterWindow / 32;
+constexpr int kFilterWarps = kBatchThreads / 32;
 
 __global__ void __launch_bounds__(kBatchThreads) filter_kernel(
     int64_t n, int64_t m, const int64_t *__restrict__ off, const float *__restrict__ score, float threshold,
     uint32_t *__restrict__ q, unsigned long long *kept) {
-    __shared__ unsigned int s_drop[kFilterWords];
-    const int tid = threadIdx.x;
+    __shared__ unsigned int s_drop_all[kFilterWarps][kFilterWords];
+    const int lane = threadIdx.x & 31;
+    unsigned int *s_drop = s_drop_all[threadIdx.x >> 5];
     auto inside = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > n ? n : x); };
-    const int64_t chunks = (m + kBatchThreads - 1) / kBatchThreads;
-    for (int64_t chunk = blockIdx.x; chunk < chunks; chunk += gridDim.x) { // block-uniform
-        const int64_t j0 = chunk * kBatchThreads, j = j0 + tid;
-        const int64_t j1 = (j0 + kBatchThreads < m) ? j0 + kBatchThreads : m;
-        int64_t a = 0, b = 0;
-        bool keep = false;
-        if (j < m) {
-            a = inside(off[j]);
-            b = inside(off[j + 1]);
-            if (b < a) b = a;
-            keep = score[j] >= threshold; // NaN: not retained
-        }
-        const int64_t A = inside(off[j0]);
-        int64_t B = inside(off[j1]);
+    const int64_t groups = (m + 31) / 32;
+    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    int64_t g = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    unsigned int kept_here = 0; // lane 0: trajectories this warp retained
+    // what the lane needs of trajectory 32 g + lane: its two offsets and its score
+    auto fetch = [&](int64_t gg, int64_t &ra, int64_t &rb, float &sc) {
+        const int64_t j = 32 * gg + lane;
+        ra = rb = 0;
+        sc = 0.f;
+        if (gg < groups && j < m) { ra = __ldg(off + j); rb = __ldg(off + j + 1); sc = __ldg(score + j); }
+    };
+    int64_t ra, rb;
+    float sc;
+    fetch(g, ra, rb, sc);
+    for (; g < groups; g += warps) { // warp-uniform
+        const int64_t j = 32 * g + lane;
+        int64_t a = inside(ra), b = inside(rb);
+        if (b < a) b = a;
+        const bool valid = j < m;
+        const bool keep = valid && sc >= threshold; // NaN: not retained
+        fetch(g + warps, ra, rb, sc);                // the next group's loads travel during the sweep
+        kept_here += __popc(__ballot_sync(0xffffffffu, keep));
+        const bool drop = valid && !keep && b > a;
+        const int last_lane = (int)min((int64_t)31, m - 1 - 32 * g);
+        const int64_t A = __shfl_sync(0xffffffffu, a, 0);
+        int64_t B = __shfl_sync(0xffffffffu, b, last_lane);
         if (B < A) B = A;
-        const int kept_here = __syncthreads_count(keep);
-        if (tid == 0 && kept && kept_here) atomicAdd(kept, (unsigned long long)kept_here);
-        const bool drop = j < m && !keep && b > a;
+        if (!__any_sync(0xffffffffu, drop)) continue; // nothing to clear in this group
         for (int64_t p = A; p < B; p += kFilterWindow) {
             const int cnt = (int)((B - p < kFilterWindow) ? B - p : kFilterWindow);
-            if (tid < kFilterWords) s_drop[tid] = 0u;
-            __syncthreads();
+            const int words = (cnt + 31) >> 5;
+            for (int wd = lane; wd < words; wd += 32) s_drop[wd] = 0u;
+            __syncwarp();
             if (drop && b > p && a < p + cnt) {
                 const int lo = (int)((a > p ? a : p) - p), hi = (int)((b < p + cnt ? b : p + cnt) - p); // [lo, hi) in [0, cnt]
                 for (int wd = lo >> 5; wd <= (hi - 1) >> 5; ++wd) {
@@ -124,12 +139,15 @@ __global__ void __launch_bounds__(kBatchThreads) filter_kernel(
                     if (DISTRL_IN(wd, kFilterWords)) atomicOr(&s_drop[wd], bits);
                 }
             }
-            __syncthreads();
-            for (int i = tid; i < cnt; i += kBatchThreads)
-                if (((s_drop[i >> 5] >> (i & 31)) & 1u) && DISTRL_IN(p + i, n)) q[p + i] = 0u;
-            __syncthreads(); // the bitmap is cleared for the next window
+            __syncwarp();
+            for (int wd = 0; wd < words; ++wd) { // 32 consecutive steps per instruction
+                const int i = 32 * wd + lane;
+                if (((s_drop[wd] >> lane) & 1u) && i < cnt && DISTRL_IN(p + i, n)) q[p + i] = 0u;
+            }
+            __syncwarp(); // the bitmap is cleared for the next window
         }
     }
+    if (lane == 0 && kept && kept_here) atomicAdd(kept, (unsigned long long)kept_here);
 }
 
 static int batch_grid(int64_t items, int64_t cap) { // cap: one resident wave of the kernel
@@ -203,7 +221,7 @@ extern "C" int distrl_filter_trajectories(int64_t n, int64_t m, const int64_t *t
     if (m == 0) return DISTRL_OK;
     if (!traj_offsets || !traj_score || (n > 0 && !prio_q)) return DISTRL_ERR_NULL;
     if (!aligned_to(traj_offsets, 8) || !aligned_to(traj_score, 4) || !aligned_to(prio_q, 4)) return DISTRL_ERR_ALIGN;
-    const int grid = batch_grid(m, one_wave_blocks(filter_kernel, kBatchThreads));
+    const int grid = batch_grid(ceil_div(m, 2), one_wave_blocks(filter_kernel, kBatchThreads)); // >= 2 groups per warp
     filter_kernel<<<grid, kBatchThreads, 0, st>>>(n, m, traj_offsets, traj_score, threshold, prio_q,
                                                   reinterpret_cast<unsigned long long *>(kept_out_device));
     DISTRL_CUDA_TRY(cudaGetLastError());
