@@ -63,3 +63,73 @@ def test_shard_zero_is_the_unsharded_workload():
         np.testing.assert_array_equal(a.arrays[k], b.arrays[k])
     c = synth.make_workload(0, shard=3)
     assert not np.array_equal(a.arrays["values"][:50], c.arrays["values"][:50])
+
+
+def _global_sampler_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import oracle
+    from paper_2410_14803_b200 import shard
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        sizes = [700, 1300, 90][:world]
+        qs = [np.random.default_rng(50 + r).integers(1, 2 ** 32, size=sizes[r], dtype=np.uint64).astype(np.uint32)
+              for r in range(world)]                                  # every rank can rebuild all shards (for the check)
+        q_local = qs[rank]
+        totals = shard.gather_totals(int(q_local.sum(dtype=np.uint64)))
+        assert totals == [int(q.sum(dtype=np.uint64)) for q in qs]
+        u = np.random.default_rng(7).integers(0, 2 ** 64, size=400, dtype=np.uint64)   # the same draws on every rank
+        u[:3] = [0, 2 ** 64 - 1, 2 ** 63]
+        owner, u_local = shard.route_draws(u.tolist(), totals)
+        mine = [j for j, g in enumerate(owner) if g == rank]
+        idx_local = oracle.sample_linear(q_local, np.array([u_local[j] for j in mine], dtype=np.uint64))
+        base = sum(sizes[:rank])
+        beta = 0.4
+        raw = oracle.is_weights(q_local, idx_local, beta, False) * shard.global_weight_factor(
+            sizes[rank], totals[rank], sum(sizes), sum(totals), beta)
+        wmax = shard.max_over_ranks([float(raw.max()) if len(mine) else 0.0])[0]
+        out.put((rank, mine, (base + idx_local).tolist(), (raw / wmax).tolist()))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_draws_routed_to_their_shards_equal_one_linear_scan_over_all_masses():
+    import oracle
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_global_sampler_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = [out.get(timeout=120) for _ in range(world)]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    sizes = [700, 1300]
+    q_all = np.concatenate([np.random.default_rng(50 + r).integers(1, 2 ** 32, size=sizes[r], dtype=np.uint64).astype(np.uint32)
+                            for r in range(world)])
+    u = np.random.default_rng(7).integers(0, 2 ** 64, size=400, dtype=np.uint64)
+    u[:3] = [0, 2 ** 64 - 1, 2 ** 63]
+    want_idx = oracle.sample_linear(q_all, u)                         # one linear scan over the concatenation
+    want_w = oracle.is_weights(q_all, want_idx, 0.4, True)
+    got_idx = np.full(400, -1, dtype=np.int64)
+    got_w = np.zeros(400)
+    for rank, mine, idx, w in results:
+        got_idx[mine] = idx
+        got_w[mine] = w
+    np.testing.assert_array_equal(got_idx, want_idx)                  # every draw owned by exactly one shard
+    np.testing.assert_allclose(got_w, want_w, rtol=1e-12)
+
+
+def test_routing_identity_on_extreme_totals():
+    sys.path.insert(0, ROOT)
+    from paper_2410_14803_b200 import shard
+    rng = np.random.default_rng(3)
+    for totals in ([1, 1, 1], [2 ** 63, 5, 2 ** 62], [7], [3, 2 ** 40 + 1]):
+        us = [0, 2 ** 64 - 1, 2 ** 63] + [int(x) for x in rng.integers(0, 2 ** 64, size=200, dtype=np.uint64)]
+        owner, ul = shard.route_draws(us, totals)
+        grand = sum(totals)
+        for u, g, up in zip(us, owner, ul):
+            y = (u * grand) >> 64
+            assert sum(totals[:g]) <= y < sum(totals[:g + 1])
+            assert (up * totals[g]) >> 64 == y - sum(totals[:g])
