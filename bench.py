@@ -523,6 +523,29 @@ def run_ours(args):
         q_f = q.clone()
         v_traj = torch.rand(w.m, dtype=torch.float32, device="cuda")       # stands in for V_traj's scores
         t_fl = timed(lambda: distrl.distrl_filter_trajectories(ins.dv["traj_offsets"], v_traj, 0.5, q_f))
+        # circular buffer of trajectories: one ingest of 512 new trajectories (their rows and masses already on the
+        # device, their lengths known on the host) into a ring of N slots with its sampler kept exact
+        ring_f = [f32() for _ in range(5)]
+        ring_q = torch.empty(n, dtype=torch.int32, device="cuda")
+        m_cap = w.m + 4096
+        ring_off = torch.empty(m_cap + 1, dtype=torch.int64, device="cuda")
+        ring_alive = torch.empty(m_cap, dtype=torch.float32, device="cuda")
+        ws_ring = distrl.alloc_workspace(distrl.distrl_replay_workspace_bytes(n))
+        rb = distrl.distrl_replay_create(ring_f, ring_q, ring_off, ring_alive, ws_ring)
+        ws_rs = distrl.alloc_workspace(distrl.distrl_sampler_workspace_bytes(n))
+        distrl.distrl_workspace_init(ws_rs)
+        s_ring = distrl.distrl_build_sampler(ring_q, ws_rs)
+        new_off = a["traj_offsets"][:513].copy()
+        rows_new = int(new_off[-1])
+        d_new_off = torch.from_numpy(new_off).cuda()
+        new_fields = [ins.dv["rewards"][:rows_new], ins.dv["values"][:rows_new], ins.lp_buf[:rows_new],
+                      ins.lm_buf[:rows_new], ins.dv["entropy"][:rows_new]]
+        new_mass = q[:rows_new].clone()
+        t_in = timed(lambda: distrl.distrl_replay_ingest(rb, s_ring, new_off, d_new_off, new_fields, new_mass))
+        if distrl.distrl_get_status(ws_ring) or distrl.distrl_get_status(ws_rs):
+            raise SystemExit("device status after the ring ingest")
+        s_ring.close()
+        rb.close()
         mc_bytes, tr_bytes = 9 * n + 8 * (w.m + 1), 16 * n + 8 * (w.m + 1) + 4 * w.m
         next_rows = {
             "mc_returns": {"ms": t_mc * 1e3, "gbs": mc_bytes / t_mc / 1e9, "frac": mc_bytes / t_mc / 1e9 / _peaks()[0]},
@@ -532,6 +555,7 @@ def run_ours(args):
                                           "frac": 16 * n / t_ca / 1e9 / _peaks()[0]},
             "actor_coefficients_batch": {"k": k, "us": t_ck * 1e6},
             "filter_trajectories": {"ms": t_fl * 1e3, "dropped_fraction": 0.5, "transitions_per_s": n / t_fl},
+            "replay_ingest": {"trajectories": 512, "rows": rows_new, "us": t_in * 1e6},
         }
         if distrl.distrl_get_status(ws_r) or distrl.distrl_get_status(ws_s):
             raise SystemExit("device status after the extra entry points")
@@ -627,7 +651,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch the sampling rounds one call at a time")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--next-rows", action="store_true",
-                    help="also time Monte-Carlo returns, trajectory-level priorities and a circular overwrite")
+                    help="also time the entry points beyond the main path, each alone on the same buffer")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -238,6 +238,15 @@ int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k, float bet
                   int normalise, int64_t *idx_out, float *is_weight_out, void *stream);
 
 /*
+ * Stratified draws (the variant of the prioritized replay the paper's DPER cites:
+ * the range of cumulative mass is cut into k equal strata and draw j is taken
+ * from stratum j).  Turns k uniforms into stratified ones,
+ *   u_out[j] = floor((j 2^64 + u_fix[j]) / k)     (0.64 fixed point; in place is fine),
+ * which are then given to distrl_sample as they are: sampling itself is unchanged.
+ */
+int distrl_stratify_uniforms(const uint64_t *u_fix, int64_t k, uint64_t *u_out, void *stream);
+
+/*
  * Priority refresh for sampled indices (Section 5.3: priorities are updated
  * from the latest policy).  For j = 0..k-1 in order:
  *   mass_j = (w_td |new_abs_delta[j]| + w_rho min(rho_i, rho_clip) + w_ent H_i)^alpha,

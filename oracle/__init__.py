@@ -242,6 +242,14 @@ def filter_trajectories(traj_offsets, traj_score, threshold, q):
                                               _d(threshold), _p(q)))
 
 
+def stratify(u):
+    """Stratified uniforms: draw j gets floor((j 2^64 + u_j) / k), i.e. a uniform from the j-th of k equal strata."""
+    u = np.ascontiguousarray(u, dtype=np.uint64)
+    out = np.empty_like(u)
+    _load().oracle_stratify(_n(u.shape[0]), _p(u), _p(out))
+    return out
+
+
 class Ring:
     """Circular replay buffer of whole trajectories (App. A "Circular Replay Buffer", Section 5.3): the
     oracle's state.  ``fields`` are the per-transition fp64 arrays, ``q`` the masses, ``alive`` / ``start``

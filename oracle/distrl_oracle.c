@@ -426,3 +426,16 @@ int64_t oracle_ring_segments(int64_t n, const uint8_t *start, const uint8_t *ali
     off_out[m] = n;
     return m;
 }
+
+/* Stratified draws of prioritized replay (Schaul et al., the replay the paper's DPER builds on): the unit
+ * interval is cut into k equal strata and draw j takes its uniform from stratum j,
+ *   u'_j = (j + u_j) / k     in 0.64 fixed point:  u'_j = floor((j 2^64 + u_j) / k),
+ * so that a batch covers the whole range of cumulative mass.  Sampling itself is unchanged. */
+int oracle_stratify(int64_t k, const uint64_t *u, uint64_t *u_out)
+{
+    for (int64_t j = 0; j < k; ++j) {
+        unsigned __int128 x = ((unsigned __int128)(uint64_t)j << 64) + u[j];
+        u_out[j] = (uint64_t)(x / (unsigned __int128)(uint64_t)k);
+    }
+    return 0;
+}

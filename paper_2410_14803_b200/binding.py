@@ -113,6 +113,7 @@ def _open(path):
         "distrl_sampler_workspace_bytes": (sz, [i64]),
         "distrl_build_sampler": (ci, [vp, i64, vp, sz, vp, ctypes.POINTER(vp)]),
         "distrl_sample": (ci, [vp, vp, i64, f32, ci, vp, vp, vp]),
+        "distrl_stratify_uniforms": (ci, [vp, i64, vp, vp]),
         "distrl_update_priorities": (ci, [vp, vp, i64, vp, vp, vp, vp, ctypes.POINTER(distrl_prio_cfg), vp, vp]),
         "distrl_retrace_priorities_build": (ci, [ctypes.POINTER(distrl_batch), f32, f32, vp, vp,
                                                  ctypes.POINTER(distrl_prio_cfg), vp, vp, vp, vp, vp, vp, sz, vp, sz, vp,
@@ -310,6 +311,14 @@ def distrl_sample(s: Sampler, u_fix, beta: float, normalise: bool, idx_out, is_w
     _check(_load().distrl_sample(s.handle, _ptr(u_fix), u_fix.numel(), beta, 1 if normalise else 0,
                                  _ptr(idx_out, torch.int64), _ptr(is_weight_out, torch.float32),
                                  _stream(stream)), "distrl_sample")
+
+
+def distrl_stratify_uniforms(u_fix: torch.Tensor, u_out: torch.Tensor, stream=None):
+    """u_out[j] = floor((j 2^64 + u_fix[j]) / k): uniforms for stratified draws (u_out may be u_fix)."""
+    if u_fix.element_size() != 8 or u_out.element_size() != 8 or u_out.numel() != u_fix.numel():
+        raise ValueError("two arrays of 64-bit fixed-point uniforms of the same length")
+    _check(_load().distrl_stratify_uniforms(_ptr(u_fix), u_fix.numel(), _ptr(u_out), _stream(stream)),
+           "distrl_stratify_uniforms")
 
 
 def distrl_update_priorities(s: Sampler, idx, new_abs_delta, logp_target, logp_behaviour, entropy,

@@ -889,6 +889,30 @@ extern "C" int distrl_replay_overwrite(distrl_sampler *s, int64_t head, int64_t 
     return DISTRL_OK;
 }
 
+namespace distrl {
+// u_out[j] = floor((j 2^64 + u[j]) / k): a uniform from the j-th of k equal strata (in place is fine)
+__global__ void stratify_kernel(const unsigned long long *__restrict__ u, long long k, unsigned long long *__restrict__ out) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < k; j += stride) {
+        const unsigned __int128 x = ((unsigned __int128)(unsigned long long)j << 64) + u[j];
+        out[j] = (unsigned long long)(x / (unsigned __int128)(unsigned long long)k);
+    }
+}
+} // namespace distrl
+
+extern "C" int distrl_stratify_uniforms(const uint64_t *u_fix, int64_t k, uint64_t *u_out, void *stream) {
+    if (k < 0 || k > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
+    if (k == 0) return DISTRL_OK;
+    if (!u_fix || !u_out) return DISTRL_ERR_NULL;
+    if (!aligned_to(u_fix, 8) || !aligned_to(u_out, 8)) return DISTRL_ERR_ALIGN;
+    int64_t grid = ceil_div(k, 256);
+    if (grid > 1184) grid = 1184;
+    stratify_kernel<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<const unsigned long long *>(u_fix), (long long)k, reinterpret_cast<unsigned long long *>(u_out));
+    DISTRL_CUDA_TRY(cudaGetLastError());
+    return DISTRL_OK;
+}
+
 extern "C" int distrl_sampler_total(distrl_sampler *s, uint64_t *total_out_device, void *stream) {
     if (!s || !total_out_device) return DISTRL_ERR_NULL;
     if (!aligned_to(total_out_device, 8)) return DISTRL_ERR_ALIGN;

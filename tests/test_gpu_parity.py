@@ -501,6 +501,46 @@ def test_two_samplers_drawing_at_the_same_time_on_two_streams():
     sb.close()
 
 
+def test_draws_over_two_shards_through_the_ordinary_entry_point():
+    # one replay over two shards (two samplers, as two GPUs would hold them): the draws routed to their owner
+    # with the exact local uniform come out of distrl_sample as one linear scan over all masses would give them
+    from paper_2410_14803_b200 import shard
+    qa, qb = _masses(300_001, 31), _masses(123_457, 32, heavy=False)
+    (sa, tqa, wsa), (sb, tqb, wsb) = _build(qa), _build(qb)
+    totals = [int(qa.sum(dtype=np.uint64)), int(qb.sum(dtype=np.uint64))]
+    u = np.random.default_rng(33).integers(0, 2 ** 64, size=3000, dtype=np.uint64)
+    owner, u_local = shard.route_draws(u.tolist(), totals)
+    got = np.full(3000, -1, dtype=np.int64)
+    for g, (s, base) in enumerate(((sa, 0), (sb, qa.shape[0]))):
+        mine = np.array([j for j, o in enumerate(owner) if o == g])
+        ul = np.array([u_local[j] for j in mine], dtype=np.uint64)
+        idx, _ = _sample(s, ul, 0.4)
+        got[mine] = base + idx
+    np.testing.assert_array_equal(got, sample_by_prefix(np.concatenate([qa, qb]), u))
+    sa.close()
+    sb.close()
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 255, 4096, 100_003])
+def test_stratified_uniforms_and_a_stratified_batch(k):
+    rng = np.random.default_rng(k)
+    u = rng.integers(0, 2 ** 64, size=k, dtype=np.uint64)
+    u[0], u[-1] = 0, 2 ** 64 - 1
+    d_u = dev(u.view(np.int64))
+    out = torch.empty_like(d_u)
+    distrl.distrl_stratify_uniforms(d_u, out)
+    want = oracle.stratify(u)
+    np.testing.assert_array_equal(out.cpu().numpy().view(np.uint64), want)
+    distrl.distrl_stratify_uniforms(d_u, d_u)                                    # in place
+    np.testing.assert_array_equal(d_u.cpu().numpy().view(np.uint64), want)
+    q = _masses(50_000, 5)
+    s, tq, ws = _build(q)
+    idx, wts = _sample(s, want, 0.4)
+    np.testing.assert_array_equal(idx, sample_by_prefix(q, want))
+    assert np.all(np.diff(idx) >= 0)                                             # one draw per stratum, in order
+    s.close()
+
+
 def test_sampling_brute_force_on_device():
     # every threshold y in [0, total) must land on index i exactly q_i times
     q = np.array([3, 1, 7, 1, 1, 12, 5] * 40, dtype=np.uint32)

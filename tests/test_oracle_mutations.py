@@ -106,6 +106,8 @@ MUTATIONS = {
         ("if (h + T > n) { advance += n - h; h = 0; }", "if (h + T > n) { h = 0; }"),
     "ring: rows are taken from the start of the call's rows for every trajectory":
         ("field[f][h + i] = new_field[f][new_off[j] + i];", "field[f][h + i] = new_field[f][i];"),
+    "stratified draws: the stratum index is not scaled to fixed point":
+        ("unsigned __int128 x = ((unsigned __int128)(uint64_t)j << 64) + u[j];", "unsigned __int128 x = (unsigned __int128)(uint64_t)j + u[j];"),
     "trajectory range ends at its own start offset":
         ("end[j] = off[idx[j] + 1];", "end[j] = off[idx[j]];"),
 }

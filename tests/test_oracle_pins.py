@@ -679,3 +679,24 @@ def test_ring_retrace_over_the_segments_equals_retrace_per_live_trajectory():
         one = oracle.retrace([0, b - a], *[f[a:b] for f in ring.fields], 0.97, 0.9)
         np.testing.assert_array_equal(vt[a:b], one[0])
         np.testing.assert_array_equal(adv[a:b], one[1])
+
+
+# ------------------------------------------------------------ stratified draws ---
+def test_stratified_uniforms_fall_into_their_strata():
+    rng = np.random.default_rng(40)
+    for k in (1, 2, 3, 7, 256, 1000):
+        u = rng.integers(0, 2 ** 64, size=k, dtype=np.uint64)
+        u[0], u[-1] = 0, 2 ** 64 - 1
+        s = oracle.stratify(u)
+        for j in range(k):
+            want = ((j << 64) + int(u[j])) // k                        # Python integers: exact
+            assert int(s[j]) == want
+            assert (j << 64) // k <= int(s[j]) < -((-((j + 1) << 64)) // k)   # stratum j: [j/k, (j+1)/k)
+    # k = 1 changes nothing; thresholds of a stratified batch increase with j
+    u = rng.integers(0, 2 ** 64, size=1, dtype=np.uint64)
+    assert oracle.stratify(u)[0] == u[0]
+    s = oracle.stratify(rng.integers(0, 2 ** 64, size=64, dtype=np.uint64))
+    assert np.all(np.diff(s.astype(object)) > 0)
+    # on equal masses a stratified batch of k = n draws hits every index exactly once
+    q = np.full(64, 5, dtype=np.uint32)
+    assert sorted(oracle.sample_linear(q, s).tolist()) == list(range(64))
