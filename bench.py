@@ -495,19 +495,33 @@ def run_ours(args):
             t1.record()
             torch.cuda.synchronize()
             return t0.elapsed_time(t1) / reps * 1e-3
+        def timed_graph(fn, per=20, reps=10):
+            # short calls: `per` of them captured into a CUDA graph (fn gets the call's number, so that it can
+            # alternate between two sets of arrays) and replayed, so that the host's launch rate does not
+            # bound the figure
+            for i in range(4):
+                fn(i)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in range(per):
+                    fn(i)
+            return timed(g.replay, reps) / per
         ins = main_set
         g_ret, lab = f32(), torch.empty(n, dtype=torch.uint8, device="cuda")
-        t_mc = timed(lambda: distrl.distrl_mc_returns(ins.batch, w.gamma, g_ret, lab, workspace=ws_r))
+        t_mc = timed_graph(lambda i: distrl.distrl_mc_returns(sets[i & 1].batch, w.gamma, g_ret, lab, workspace=ws_r))
         q_traj = torch.empty(w.m, dtype=torch.int32, device="cuda")
-        t_tr = timed(lambda: distrl.distrl_compute_priorities_traj(ins.dv["traj_offsets"], prio_in, ins.lp_buf, ins.lm_buf,
-                                                                   ins.dv["entropy"], cfg, None, q_traj))
+        t_tr = timed_graph(lambda i: distrl.distrl_compute_priorities_traj(
+            sets[i & 1].dv["traj_offsets"], prio_in, sets[i & 1].lp_buf, sets[i & 1].lm_buf, sets[i & 1].dv["entropy"],
+            cfg, None, q_traj))
         s_tmp = distrl.distrl_build_sampler(q, ws_s)
         k_over = min(1 << 20, n)
         new_q = torch.randint(1, 1 << 24, (k_over,), dtype=torch.int32, device="cuda")
-        t_ov = timed(lambda: distrl.distrl_replay_overwrite(s_tmp, n - k_over // 2, new_q))
+        t_ov = timed_graph(lambda i: distrl.distrl_replay_overwrite(s_tmp, n - k_over // 2, new_q))
         s_tmp.close()
         coef_all, coef_k = f32(), torch.empty(k, dtype=torch.float32, device="cuda")
-        t_ca = timed(lambda: distrl.distrl_actor_coefficients(ins.lp_buf, ins.lm_buf, adv, coef_all))
+        t_ca = timed_graph(lambda i: distrl.distrl_actor_coefficients(sets[i & 1].lp_buf, sets[i & 1].lm_buf,
+                                                                      (adv, vt)[i & 1], coef_all))   # vt: a second array of advantages' size
         # one drawn batch: 20 calls (one per round's batch) replayed from a CUDA graph, so that the
         # figure is the device's and not the Python caller's
         def coef_batches():
@@ -520,9 +534,11 @@ def run_ours(args):
         with torch.cuda.graph(g_ck):
             coef_batches()
         t_ck = timed(g_ck.replay) / 20
-        q_f = q.clone()
-        v_traj = torch.rand(w.m, dtype=torch.float32, device="cuda")       # stands in for V_traj's scores
-        t_fl = timed(lambda: distrl.distrl_filter_trajectories(ins.dv["traj_offsets"], v_traj, 0.5, q_f))
+        # two sets of offsets, scores and masses (168 MB together, more than L2), taken in turn
+        q_f = [q.clone(), q.clone()]
+        v_traj = [torch.rand(w.m, dtype=torch.float32, device="cuda") for _ in range(2)]   # stand in for V_traj's scores
+        t_fl = timed_graph(lambda i: distrl.distrl_filter_trajectories(sets[i & 1].dv["traj_offsets"], v_traj[i & 1], 0.5,
+                                                                       q_f[i & 1]))
         # circular buffer of trajectories: one ingest of 512 new trajectories (their rows and masses already on the
         # device, their lengths known on the host) into a ring of N slots with its sampler kept exact
         ring_f = [f32() for _ in range(5)]
@@ -554,7 +570,9 @@ def run_ours(args):
             "actor_coefficients_buffer": {"ms": t_ca * 1e3, "gbs": 16 * n / t_ca / 1e9,
                                           "frac": 16 * n / t_ca / 1e9 / _peaks()[0]},
             "actor_coefficients_batch": {"k": k, "us": t_ck * 1e6},
-            "filter_trajectories": {"ms": t_fl * 1e3, "dropped_fraction": 0.5, "transitions_per_s": n / t_fl},
+            "filter_trajectories": {"ms": t_fl * 1e3, "dropped_fraction": 0.5, "transitions_per_s": n / t_fl,
+                                    "gbs": (8 * (w.m + 1) + 4 * w.m + 2 * n) / t_fl / 1e9,   # offsets, scores, zeros over half the steps
+                                    "frac": (8 * (w.m + 1) + 4 * w.m + 2 * n) / t_fl / 1e9 / _peaks()[0]},
             "replay_ingest": {"trajectories": 512, "rows": rows_new, "us": t_in * 1e6},
         }
         if distrl.distrl_get_status(ws_r) or distrl.distrl_get_status(ws_s):

@@ -147,20 +147,80 @@ __global__ void __launch_bounds__(256) build_leaf_kernel(Tree t, int vec_ok) {
     }
 }
 
-// build, pass 2: levels 3.. from level 2, one block; one warp per entry (32 children, one coalesced
-// load).  Launched with programmatic stream serialisation: it is scheduled while pass 1 drains.
-__global__ void __launch_bounds__(1024) build_upper_kernel(Tree t) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    grid_dependency_wait();
-    for (int l = 3; l <= t.levels; ++l) {
-        for (int64_t e = warp; e < t.count[l]; e += 32) {
+// build, pass 2: levels 3.. from level 2, one block, launched with programmatic stream serialisation
+// (it is scheduled while pass 1 drains).
+// Levels 3 .. levels of the tree from level 2, by the THREADS threads of one block (tid = 0 .. THREADS-1;
+// `sync` is a barrier over exactly those threads, `s_lvl` 2 x 128 words of their shared memory).  While a
+// level has more than 4096 entries: one warp per parent (32 children, one coalesced load).  From there on
+// a single round trip to global memory: every thread loads 4096 / THREADS consecutive children, the
+// neighbouring threads that share a parent add up with shuffles, and the levels above (at most 128
+// entries) are summed out of shared memory.  Level arrays are 256-byte aligned and padded.
+template <int THREADS, typename Sync>
+__device__ __forceinline__ void tree_build_upper(const Tree &t, int tid, unsigned long long (*s_lvl)[128], Sync sync) {
+    static_assert(THREADS == 128 || THREADS == 256 || THREADS == 512 || THREADS == 1024, "2 .. 32 children per thread");
+    constexpr int kPer = 4096 / THREADS;      // children per thread
+    constexpr int kShare = kFan / kPer;   // threads per parent
+    const int lane = tid & 31, warp = tid >> 5;
+    auto warp_sum = [](unsigned long long v) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+        return v;
+    };
+    int l = 3;
+    for (; l <= t.levels && t.count[l - 1] > 4096; ++l) {
+        for (int64_t e = warp; e < t.count[l]; e += THREADS / 32) {
             const int64_t ch = e * kFan + lane;
-            unsigned long long v = (ch < t.count[l - 1]) ? __ldcg(&t.lvl[l - 1][ch]) : 0ull;
-            v = warp_sum_u64(v);
-            if (lane == 0) t.lvl[l][e] = v;
+            unsigned long long v = (ch < t.count[l - 1] && DISTRL_IN(ch, t.count[l - 1])) ? __ldcg(&t.lvl[l - 1][ch]) : 0ull;
+            v = warp_sum(v);
+            if (lane == 0 && DISTRL_IN(e, t.count[l])) t.lvl[l][e] = v;
         }
-        __syncthreads();
+        sync();
     }
+    if (l > t.levels) return;
+    int cur = 0;
+    {
+        const int64_t c = t.count[l - 1];
+        const unsigned long long *src = t.lvl[l - 1] + (int64_t)kPer * tid;
+        unsigned long long v = 0ull;
+        if ((int64_t)kPer * tid + kPer <= c) {
+            ulonglong2 x[kPer / 2];
+#pragma unroll
+            for (int e = 0; e < kPer / 2; ++e) x[e] = __ldcg(reinterpret_cast<const ulonglong2 *>(src) + e);
+#pragma unroll
+            for (int e = 0; e < kPer / 2; ++e) v += x[e].x + x[e].y;
+        } else {
+#pragma unroll
+            for (int e = 0; e < kPer; ++e)
+                if ((int64_t)kPer * tid + e < c && DISTRL_IN(kPer * tid + e, c)) v += __ldcg(src + e);
+        }
+#pragma unroll
+        for (int d = kShare / 2; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+        if ((tid % kShare) == 0) {
+            s_lvl[cur][tid / kShare] = v; // zero beyond the level's last entry
+            if (tid / kShare < t.count[l] && DISTRL_IN(tid / kShare, t.count[l])) t.lvl[l][tid / kShare] = v;
+        }
+        sync();
+    }
+    for (++l; l <= t.levels; ++l) { // at most 128 children left: one warp per parent
+        const int64_t c = t.count[l - 1];
+        if (warp < t.count[l]) {
+            const int ch = warp * kFan + lane;
+            unsigned long long v = (ch < c && ch < 128) ? s_lvl[cur][ch] : 0ull;
+            v = warp_sum(v);
+            if (lane == 0) {
+                s_lvl[cur ^ 1][warp] = v;
+                if (DISTRL_IN(warp, t.count[l])) t.lvl[l][warp] = v;
+            }
+        }
+        sync();
+        cur ^= 1;
+    }
+}
+constexpr int kUpperThreads = 1024;
+__global__ void __launch_bounds__(kUpperThreads) build_upper_kernel(Tree t) {
+    __shared__ unsigned long long s_lvl[2][128];
+    grid_dependency_wait();
+    tree_build_upper<kUpperThreads>(t, (int)threadIdx.x, s_lvl, [] { __syncthreads(); });
 }
 
 __global__ void total_kernel(Tree t, unsigned long long *out) {
@@ -741,7 +801,7 @@ void sampler_tree_base(const distrl_sampler *s, TreeBase *out) {
 
 int sampler_build_upper(const distrl_sampler *s, cudaStream_t st) {
     if (s->tree.levels >= 3) {
-        DISTRL_CUDA_TRY(launch_pdl(build_upper_kernel, dim3(1), dim3(1024), 0, st, s->tree));
+        DISTRL_CUDA_TRY(launch_pdl(build_upper_kernel, dim3(1), dim3(kUpperThreads), 0, st, s->tree));
     }
     return DISTRL_OK;
 }

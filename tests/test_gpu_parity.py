@@ -1178,6 +1178,34 @@ def test_no_draw_returns_a_filtered_transition():
     s.close()
 
 
+@pytest.mark.parametrize("lead", [1, 2, 3])
+def test_filter_trajectories_mass_array_off_a_16_byte_boundary(lead):
+    # the sweep stores 16 bytes where four neighbouring steps go: the array may start anywhere on a 4-byte boundary,
+    # and nothing before or after it may be touched
+    rng = np.random.default_rng(50 + lead)
+    lens = rng.integers(0, 40, size=3000)
+    lens[::97] = 5000                                       # longer than a window
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    n, m = int(off[-1]), lens.shape[0]
+    q = rng.integers(1, 1 << 32, size=n, dtype=np.uint64).astype(np.uint32)
+    score = rng.uniform(0, 1, m).astype(np.float32)
+    score[0] = score[-1] = 0.0                              # the first and the last trajectory go
+    guard = 8
+    whole = torch.full((lead + n + guard,), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    tq = whole[lead:lead + n]
+    tq.copy_(dev(q.view(np.int32)))
+    assert tq.data_ptr() % 16 == 4 * lead
+    kept = torch.zeros(1, dtype=torch.int64, device="cuda")
+    distrl.distrl_filter_trajectories(dev(off), dev(score), 0.5, tq, kept)
+    torch.cuda.synchronize()
+    ref = q.copy()
+    kept_ref = oracle.filter_trajectories(off, score, 0.5, ref)
+    np.testing.assert_array_equal(tq.cpu().numpy().view(np.uint32), ref)
+    assert kept.item() == kept_ref
+    h = whole.cpu().numpy()
+    assert np.all(h[:lead] == 0x5A5A5A5A) and np.all(h[lead + n:] == 0x5A5A5A5A)
+
+
 def test_filter_trajectories_edges():
     from paper_2410_14803_b200 import binding
     off = np.array([0, 3, 3, 8], dtype=np.int64)
