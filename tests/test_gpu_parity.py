@@ -75,6 +75,30 @@ def test_retrace_bootstrap_values_layouts(kind, n):
     check_retrace(off, r, V, lp, lm, 0.97, 0.9, boot=boot)
 
 
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_retrace_bootstrap_values_empty_trajectories_everywhere(seed):
+    # The pipelined kernel finds the trajectory of an end from the trajectory of the lowest end in the same
+    # 32-step word of the end mask; empty trajectories break that count and are resolved by a search in the
+    # offsets.  Here they sit wherever the bookkeeping changes hands: at the start and the end of the buffer,
+    # in runs, between ends of one word, on both sides of every 2048th trajectory (one block of the mask
+    # kernel takes 2048), right after a tile boundary.
+    rng = np.random.default_rng(700 + seed)
+    m = 3 * 2048 + 777
+    lens = rng.integers(1, 6 if seed < 2 else 40, size=m)
+    lens[rng.random(m) < 0.15] = 0
+    for g in (0, 1, 2, m - 1, m - 2):
+        lens[g] = 0
+    for c in (2048, 4096, 6144):
+        lens[c - 2:c + 3] = [0, 1, 0, 0, 2][:5] if seed != 1 else [1, 0, 0, 1, 0]
+    lens[100:140] = 0                                     # a long run of empty trajectories
+    lens[140:200] = 1                                     # then an end at every step
+    lens[200:230:2] = 0
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    r, V, lp, lm = random_batch(seed + 30, off)
+    boot = rng.normal(0, 2, m).astype(np.float32)
+    check_retrace(off, r, V, lp, lm, 0.97, 0.9, boot=boot)
+
+
 def test_retrace_bootstrap_values_through_the_general_kernel():
     # arrays that are not 16-byte aligned; and a workspace without room for what the pipelined kernel
     # keeps of the bootstrap values (the fixed array of the workspace-free entry point is one)
