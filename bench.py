@@ -510,6 +510,12 @@ def run_ours(args):
         ins = main_set
         g_ret, lab = f32(), torch.empty(n, dtype=torch.uint8, device="cuda")
         t_mc = timed_graph(lambda i: distrl.distrl_mc_returns(sets[i & 1].batch, w.gamma, g_ret, lab, workspace=ws_r))
+        # Retrace with a bootstrap value per trajectory (the pipelined kernel's other instance)
+        boot_v = torch.rand(w.m, dtype=torch.float32, device="cuda")
+        boot_batches = [distrl.make_batch(x.dv["traj_offsets"], x.dv["rewards"], x.dv["values"], x.lp_buf, x.lm_buf, boot_v)
+                        for x in sets]
+        t_bt = timed_graph(lambda i: distrl.distrl_retrace_targets(boot_batches[i & 1], w.gamma, w.lam, vt, adv, dl,
+                                                                   workspace=ws_r))
         q_traj = torch.empty(w.m, dtype=torch.int32, device="cuda")
         t_tr = timed_graph(lambda i: distrl.distrl_compute_priorities_traj(
             sets[i & 1].dv["traj_offsets"], prio_in, sets[i & 1].lp_buf, sets[i & 1].lm_buf, sets[i & 1].dv["entropy"],
@@ -563,8 +569,10 @@ def run_ours(args):
         s_ring.close()
         rb.close()
         mc_bytes, tr_bytes = 9 * n + 8 * (w.m + 1), 16 * n + 8 * (w.m + 1) + 4 * w.m
+        bt_bytes = 28 * n + 8 * (w.m + 1) + 4 * w.m      # the Retrace call's bytes and one bootstrap value per trajectory
         next_rows = {
             "mc_returns": {"ms": t_mc * 1e3, "gbs": mc_bytes / t_mc / 1e9, "frac": mc_bytes / t_mc / 1e9 / _peaks()[0]},
+            "retrace_bootstrap": {"ms": t_bt * 1e3, "gbs": bt_bytes / t_bt / 1e9, "frac": bt_bytes / t_bt / 1e9 / _peaks()[0]},
             "priorities_traj": {"ms": t_tr * 1e3, "gbs": tr_bytes / t_tr / 1e9, "frac": tr_bytes / t_tr / 1e9 / _peaks()[0]},
             "replay_overwrite": {"slots": k_over, "ms": t_ov * 1e3, "slots_per_s": k_over / t_ov},
             "actor_coefficients_buffer": {"ms": t_ca * 1e3, "gbs": 16 * n / t_ca / 1e9,
