@@ -341,7 +341,7 @@ def run_ours(args):
     ev = lambda: torch.cuda.Event(enable_timing=True)
     # a refresh of up to 8192 positions is one launch, a longer one a claim and an apply launch per 65536 positions
     per_round = 1 + (1 if (k <= 8192 and n < 2 ** 31) else 2 * ((k + 65535) // 65536))
-    retrace_launches = 4 if tok else 2   # end mask + scan (token-level: + the two stand-ins for dense buffers)
+    retrace_launches = 5 if tok else 2   # end mask + scan (token-level: + the dense instance and the general pair, which return at once)
     launches_per_step = retrace_launches + 1 + 2 + per_round * R   # Retrace, priorities, 2 build, (sample, refresh) x R
     if args.fused:
         launches_per_step = 3 + per_round * R       # end mask + fused scan + upper tree levels, then the rounds
@@ -618,7 +618,7 @@ def run_ours(args):
                        "build_sampler": None if args.fused else float(stage_min[2]), "rounds": float(stage_min[3])},
             "timed_steps": int(args.steps),
         },
-        "roofline": {"bound": "hbm", "kernel": ("scan_mask_kernel + scan_pipe_kernel<fused> (distrl_retrace_priorities_build)" if args.fused else "scan_mask_kernel + %s (distrl_retrace_targets)" % ("scan_tok_pipe_kernel (+ two stand-ins that return at once)" if tok else "scan_pipe_kernel")), "achieved": ach, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": ("scan_mask_kernel + scan_pipe_kernel<fused> (distrl_retrace_priorities_build)" if args.fused else "scan_mask_kernel + %s (distrl_retrace_targets)" % ("scan_tok_pipe_kernel (+ three stand-ins for dense buffers that return at once)" if tok else "scan_pipe_kernel")), "achieved": ach, "peak": peak,
                      "unit": "GB/s", "frac": ach / peak, "peak_kind": "of " + peak_kind,
                      "frac_of_nominal_8000": ach / 8000.0, "traffic": _measured_traffic(w.name) if (args.n_override is None and not args.fused) else None,
                      "algorithmic_bytes": retrace_bytes},

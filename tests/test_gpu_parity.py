@@ -730,6 +730,21 @@ def test_token_level_tile_edges(n, kind):
     _token_case(off, sto, tok_p, tok_m, n)
 
 
+@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 511, 512, 513, 544, 545, 546, 1023, 1024, 1025, 1057, 1569, 4097, 40001])
+@pytest.mark.parametrize("kind", ["single", "ones", "tile_straddle", "long_mixed"])
+def test_token_level_tile_edges_dense_instance(n, kind):
+    # the same sizes with 18 to 40 tokens per step: the instance with one step per lane and sixteen token warps
+    rng = np.random.default_rng(2000 + n)
+    cnt = rng.integers(18, 41, n)
+    cnt[rng.random(n) < 0.05] = 0
+    sto = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int64)
+    nt = int(sto[-1])
+    tok_m = synth.f32_to_bf16_bits((rng.standard_normal(nt) * 0.3 - 0.3).astype(np.float32) / np.float32(2))
+    tok_p = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(tok_m) + (rng.standard_normal(nt) * 0.05).astype(np.float32))
+    off = synth.adversarial_offsets(kind, n, tile=512)
+    _token_case(off, sto, tok_p, tok_m, n)
+
+
 @pytest.mark.parametrize("counts", ["first_vector_only", "sparse", "near_capacity", "over_capacity_some"])
 def test_token_level_staging_corners(counts):
     # first_vector_only: all tokens of a tile inside one 16-byte vector; sparse: most steps empty;
@@ -748,10 +763,11 @@ def test_token_level_staging_corners(counts):
     _token_case(off, sto, tok_p, tok_m, 5)
 
 
-@pytest.mark.parametrize("lo,hi", [(20, 33), (17, 19), (16, 18)])
+@pytest.mark.parametrize("lo,hi", [(20, 33), (17, 19), (16, 18), (32, 36), (34, 36), (36, 48), (0, 70)])
 def test_token_level_dense_buffers(lo, hi):
-    # mean token counts around and above what a stage of the pipelined kernel holds (about 17 per step):
-    # the call hands dense buffers to the general kernel; either way the results are the oracle's
+    # mean token counts around and above what a stage of the pipelined kernel holds (about 17 per step) and what
+    # a stage of its instance for dense buffers holds (about 34): the mask kernel's verdict on the mean sends the
+    # call to one of them or to the general kernel; whichever it is, the results are the oracle's
     n = 120001
     rng = np.random.default_rng(lo * 100 + hi)
     cnt = rng.integers(lo, hi, n)
@@ -782,23 +798,25 @@ def test_token_level_bad_step_offsets_are_reported_not_fatal():
     assert good["status"] == 0
 
 
-@pytest.mark.parametrize("pattern", ["workload", "alternating"])
+@pytest.mark.parametrize("pattern", ["workload", "alternating", "dense_alternating"])
 def test_token_level_repeated_runs_agree_bit_for_bit(pattern):
     # The token kernel's warps hand data to one another through shared-memory buffers guarded by
     # mbarriers, and drift apart by up to a tile: forty runs on the same inputs and workspace must
     # agree bit for bit.  "alternating": tiles of one token per step alternate with tiles of 17, so
-    # that the same shared-memory positions belong to different warps in consecutive tiles.
+    # that the same shared-memory positions belong to different warps in consecutive tiles;
+    # "dense_alternating": tiles of 12 and of 36 tokens per step, which the instance for dense buffers takes.
     if pattern == "workload":
         w = synth.make_workload(4, n_override=1500001)
         a = w.arrays
         n, off, sto, tp, tm = w.n, a["traj_offsets"], a["step_token_offsets"], a["tok_logp_target"], a["tok_logp_behaviour"]
     else:
-        n = 1200000
+        n = 1200000 if pattern == "alternating" else 600000
         rng = np.random.default_rng(12)
-        cnt = np.where((np.arange(n) // 512) % 2 == 0, 1, 17)
+        cnt = np.where((np.arange(n) // 512) % 2 == 0, 1, 17) if pattern == "alternating" else \
+            np.where((np.arange(n) // 512) % 2 == 0, 12, 36)
         sto = np.concatenate([[0], np.cumsum(cnt)]).astype(np.int64)
         nt = int(sto[-1])
-        tm = synth.f32_to_bf16_bits((rng.standard_normal(nt) * 0.3 - 0.3).astype(np.float32))
+        tm = synth.f32_to_bf16_bits((rng.standard_normal(nt) * 0.3 - 0.3).astype(np.float32) / np.float32(2))
         tp = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(tm) + (rng.standard_normal(nt) * 0.05).astype(np.float32))
         off = synth.adversarial_offsets("long_mixed", n, tile=512)
     rng = np.random.default_rng(8)
