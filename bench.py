@@ -516,6 +516,23 @@ def run_ours(args):
                         for x in sets]
         t_bt = timed_graph(lambda i: distrl.distrl_retrace_targets(boot_batches[i & 1], w.gamma, w.lam, vt, adv, dl,
                                                                    workspace=ws_r))
+        # token-level Retrace on a dense buffer (32 tokens per step, 8 M steps, trajectories of 10 steps): the
+        # instance of the pipelined token kernel with one step per lane
+        nd, per = 8_000_000, 32
+        d_sto = torch.arange(0, (nd + 1) * per, per, dtype=torch.int64, device="cuda")
+        d_tm = torch.randn(nd * per, device="cuda").mul_(0.3).sub_(0.3).to(torch.bfloat16)
+        d_tp = (d_tm.float() + torch.randn(nd * per, device="cuda") * 0.05).to(torch.bfloat16)
+        d_off = torch.arange(0, nd + 1, 10, dtype=torch.int64, device="cuda")
+        d_r, d_v = torch.randn(nd, device="cuda"), torch.rand(nd, device="cuda")
+        d_batch = distrl.make_batch(d_off, d_r, d_v, None, None, None, d_sto, d_tp, d_tm)
+        d_out = [torch.empty(nd, dtype=torch.float32, device="cuda") for _ in range(5)]
+        ws_d = distrl.alloc_workspace(distrl.distrl_retrace_workspace_bytes(nd))
+        distrl.distrl_workspace_init(ws_d)
+        t_td = timed_graph(lambda i: distrl.distrl_retrace_targets(d_batch, w.gamma, w.lam, *d_out, workspace=ws_d), per=5)
+        if distrl.distrl_get_status(ws_d):
+            raise SystemExit("device status after the dense token-level call")
+        td_bytes = 36 * nd + 4 * nd * per + 8 * (nd // 10 + 1)
+        del d_tm, d_tp, d_out
         q_traj = torch.empty(w.m, dtype=torch.int32, device="cuda")
         t_tr = timed_graph(lambda i: distrl.distrl_compute_priorities_traj(
             sets[i & 1].dv["traj_offsets"], prio_in, sets[i & 1].lp_buf, sets[i & 1].lm_buf, sets[i & 1].dv["entropy"],
@@ -573,6 +590,8 @@ def run_ours(args):
         next_rows = {
             "mc_returns": {"ms": t_mc * 1e3, "gbs": mc_bytes / t_mc / 1e9, "frac": mc_bytes / t_mc / 1e9 / _peaks()[0]},
             "retrace_bootstrap": {"ms": t_bt * 1e3, "gbs": bt_bytes / t_bt / 1e9, "frac": bt_bytes / t_bt / 1e9 / _peaks()[0]},
+            "retrace_tokens_dense": {"steps": nd, "tokens_per_step": per, "ms": t_td * 1e3, "gbs": td_bytes / t_td / 1e9,
+                                     "frac": td_bytes / t_td / 1e9 / _peaks()[0]},
             "priorities_traj": {"ms": t_tr * 1e3, "gbs": tr_bytes / t_tr / 1e9, "frac": tr_bytes / t_tr / 1e9 / _peaks()[0]},
             "replay_overwrite": {"slots": k_over, "ms": t_ov * 1e3, "slots_per_s": k_over / t_ov},
             "actor_coefficients_buffer": {"ms": t_ca * 1e3, "gbs": 16 * n / t_ca / 1e9,
