@@ -90,9 +90,9 @@ int distrl_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
  *   delta_t = r_t + gamma V(s_{t+1}) - V(s_t)
  *   Delta_t = sum_{k>=t} gamma^(k-t) (prod_{i=t+1..k} c_i) delta_k   (per trajectory)
  *   v_target_t = V(s_t) + Delta_t;  advantage_t = Delta_t;  td_delta_t = delta_t
- * V(s_{t+1}) of a trajectory's last step is bootstrap_values[j], or 0.  (With
- * bootstrap values the call uses `advantage` as scratch before it writes the
- * results there; like every output it must not alias an input.)
+ * V(s_{t+1}) of a trajectory's last step is bootstrap_values[j], or 0.  (The
+ * bootstrap values are read in place while the outputs are written: like every
+ * input the array must not alias an output.)
  * Computed in fp32 as a segmented reverse scan; results agree with fp64
  * evaluation of the definition to 1e-4 (1 + |ref|).
  *   v_target, advantage : [N] outputs, required.
