@@ -80,23 +80,27 @@ __global__ void __launch_bounds__(kBatchThreads) traj_ranges_kernel(
 }
 
 // Trajectory filter: a warp takes 32 consecutive trajectories, whose steps are one contiguous range of
-// the buffer, and walks that range in windows of kFilterWindow steps.  Per window the lane of every
-// trajectory that is not retained sets the bits of its steps in the warp's own bitmap in shared memory
-// (whole words at a time), then the warp sweeps the window, 32 consecutive steps per instruction, with
-// coalesced stores of zero where a bit is set.  Masses of retained trajectories are neither read nor
-// written.  Warps never meet at a block barrier; the loads of the next group of trajectories are sent
-// for before the current one is swept.
-constexpr int kFilterWindow = 2048;
-constexpr int kFilterWords = kFilterWindow / 32;
+// the buffer, and walks that range in windows of kFilterWindow steps, one 32-step word per lane.  Per
+// window the lane of every trajectory that is not retained toggles two bits in the warp's own 128
+// bytes of shared memory, one where its steps begin and one where they end (neighbouring dropped
+// trajectories cancel at their common boundary); a running parity over the bits then marks exactly the
+// steps to clear: inside each word by five shift-and-XOR steps, across words by one ballot.  The warp
+// sweeps the window, 32 consecutive steps per instruction, with coalesced stores of zero where a bit is
+// set.  Masses of retained trajectories are neither read nor written.  Warps never meet at a block
+// barrier; the loads of the next group of trajectories are sent for before the current one is swept.
+// I is the type of a position in the buffer: int when n < 2^31.
+constexpr int kFilterWindow = 1024;
 constexpr int kFilterWarps = kBatchThreads / 32;
 
+template <typename I>
 __global__ void __launch_bounds__(kBatchThreads) filter_kernel(
-    int64_t n, int64_t m, const int64_t *__restrict__ off, const float *__restrict__ score, float threshold,
+    int64_t n64, int64_t m, const int64_t *__restrict__ off, const float *__restrict__ score, float threshold,
     uint32_t *__restrict__ q, unsigned long long *kept) {
-    __shared__ unsigned int s_drop_all[kFilterWarps][kFilterWords];
+    __shared__ unsigned int s_tog_all[kFilterWarps][32];
     const int lane = threadIdx.x & 31;
-    unsigned int *s_drop = s_drop_all[threadIdx.x >> 5];
-    auto inside = [&](int64_t x) { return x < 0 ? (int64_t)0 : (x > n ? n : x); };
+    unsigned int *s_tog = s_tog_all[threadIdx.x >> 5];
+    const I n = (I)n64;
+    auto inside = [&](int64_t x) { return x < 0 ? (I)0 : (x > n64 ? n : (I)x); };
     const int64_t groups = (m + 31) / 32;
     const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     int64_t g = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -113,7 +117,8 @@ __global__ void __launch_bounds__(kBatchThreads) filter_kernel(
     fetch(g, ra, rb, sc);
     for (; g < groups; g += warps) { // warp-uniform
         const int64_t j = 32 * g + lane;
-        int64_t a = inside(ra), b = inside(rb);
+        const I a = inside(ra);
+        I b = inside(rb);
         if (b < a) b = a;
         const bool valid = j < m;
         const bool keep = valid && sc >= threshold; // NaN: not retained
@@ -121,30 +126,37 @@ __global__ void __launch_bounds__(kBatchThreads) filter_kernel(
         kept_here += __popc(__ballot_sync(0xffffffffu, keep));
         const bool drop = valid && !keep && b > a;
         const int last_lane = (int)min((int64_t)31, m - 1 - 32 * g);
-        const int64_t A = __shfl_sync(0xffffffffu, a, 0);
-        int64_t B = __shfl_sync(0xffffffffu, b, last_lane);
+        const I A = __shfl_sync(0xffffffffu, a, 0);
+        I B = __shfl_sync(0xffffffffu, b, last_lane);
         if (B < A) B = A;
         if (!__any_sync(0xffffffffu, drop)) continue; // nothing to clear in this group
-        for (int64_t p = A; p < B; p += kFilterWindow) {
-            const int cnt = (int)((B - p < kFilterWindow) ? B - p : kFilterWindow);
+        for (I p = A; p < B; p += kFilterWindow) {
+            // positions inside a window fit 32 bits: everything below is relative to p
+            const int cnt = (int)((B - p < (I)kFilterWindow) ? B - p : (I)kFilterWindow);
+            s_tog[lane] = 0u;
+            __syncwarp();
+            if (drop && b > p && a - p < (I)cnt) {
+                const int lo = (a > p) ? (int)(a - p) : 0;                                  // in [0, cnt)
+                const int hi = (b - p < (I)cnt) ? (int)(b - p) : kFilterWindow;            // in (lo, cnt) or "to the end"
+                atomicXor(&s_tog[lo >> 5], 1u << (lo & 31));
+                if (hi < kFilterWindow) atomicXor(&s_tog[hi >> 5], 1u << (hi & 31));
+            }
+            __syncwarp();
+            // running parity: a step is cleared iff an odd number of toggles lies at or before it
+            unsigned int x = s_tog[lane];
+            x ^= x << 1; x ^= x << 2; x ^= x << 4; x ^= x << 8; x ^= x << 16;
+            const unsigned int odd = __ballot_sync(0xffffffffu, x >> 31);    // words that end inside a run
+            if (__popc(odd & ((1u << lane) - 1u)) & 1) x = ~x;                // the run of the words before goes on
+            // a run that reaches the window's end was left open: nothing beyond the last step
+            const int tail = cnt - 32 * lane;
+            x = tail >= 32 ? x : (tail > 0 ? x & ((1u << tail) - 1u) : 0u);
             const int words = (cnt + 31) >> 5;
-            for (int wd = lane; wd < words; wd += 32) s_drop[wd] = 0u;
-            __syncwarp();
-            if (drop && b > p && a < p + cnt) {
-                const int lo = (int)((a > p ? a : p) - p), hi = (int)((b < p + cnt ? b : p + cnt) - p); // [lo, hi) in [0, cnt]
-                for (int wd = lo >> 5; wd <= (hi - 1) >> 5; ++wd) {
-                    const int first = (wd == (lo >> 5)) ? (lo & 31) : 0;
-                    const int last = (wd == ((hi - 1) >> 5)) ? ((hi - 1) & 31) : 31; // inclusive
-                    const unsigned int bits = (0xFFFFFFFFu >> (31 - last)) & (0xFFFFFFFFu << first);
-                    if (DISTRL_IN(wd, kFilterWords)) atomicOr(&s_drop[wd], bits);
-                }
-            }
-            __syncwarp();
+            uint32_t *const qp = q + p + lane;
             for (int wd = 0; wd < words; ++wd) { // 32 consecutive steps per instruction
-                const int i = 32 * wd + lane;
-                if (((s_drop[wd] >> lane) & 1u) && i < cnt && DISTRL_IN(p + i, n)) q[p + i] = 0u;
+                const unsigned int mw = __shfl_sync(0xffffffffu, x, wd);
+                if (((mw >> lane) & 1u) && DISTRL_IN((int64_t)p + 32 * wd + lane, n64)) qp[32 * wd] = 0u;
             }
-            __syncwarp(); // the bitmap is cleared for the next window
+            __syncwarp(); // the toggles are cleared for the next window
         }
     }
     if (lane == 0 && kept && kept_here) atomicAdd(kept, (unsigned long long)kept_here);
@@ -221,9 +233,15 @@ extern "C" int distrl_filter_trajectories(int64_t n, int64_t m, const int64_t *t
     if (m == 0) return DISTRL_OK;
     if (!traj_offsets || !traj_score || (n > 0 && !prio_q)) return DISTRL_ERR_NULL;
     if (!aligned_to(traj_offsets, 8) || !aligned_to(traj_score, 4) || !aligned_to(prio_q, 4)) return DISTRL_ERR_ALIGN;
-    const int grid = batch_grid(ceil_div(m, 2), one_wave_blocks(filter_kernel, kBatchThreads)); // >= 2 groups per warp
-    filter_kernel<<<grid, kBatchThreads, 0, st>>>(n, m, traj_offsets, traj_score, threshold, prio_q,
-                                                  reinterpret_cast<unsigned long long *>(kept_out_device));
+    if (n < ((int64_t)1 << 31) - kFilterWindow) {
+        const int grid = batch_grid(ceil_div(m, 2), one_wave_blocks(filter_kernel<int>, kBatchThreads)); // >= 2 groups per warp
+        filter_kernel<int><<<grid, kBatchThreads, 0, st>>>(n, m, traj_offsets, traj_score, threshold, prio_q,
+                                                           reinterpret_cast<unsigned long long *>(kept_out_device));
+    } else {
+        const int grid = batch_grid(ceil_div(m, 2), one_wave_blocks(filter_kernel<int64_t>, kBatchThreads));
+        filter_kernel<int64_t><<<grid, kBatchThreads, 0, st>>>(n, m, traj_offsets, traj_score, threshold, prio_q,
+                                                               reinterpret_cast<unsigned long long *>(kept_out_device));
+    }
     DISTRL_CUDA_TRY(cudaGetLastError());
     return DISTRL_OK;
 }
