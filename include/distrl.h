@@ -247,6 +247,49 @@ int distrl_sample(distrl_sampler *s, const uint64_t *u_fix, int64_t k, float bet
 int distrl_stratify_uniforms(const uint64_t *u_fix, int64_t k, uint64_t *u_out, void *stream);
 
 /*
+ * One prioritized replay over several shards (one per GPU): the proportional
+ * draw of App. A ("Priority-Based Sampling": P(i) = p_i^alpha / sum_j p_j^alpha)
+ * taken over the concatenation of the shards' masses.  Draw j has the global
+ * threshold y = floor(u_fix[j] T / 2^64), T the sum of shard_totals; it belongs to
+ * the shard whose range of cumulative mass holds y, and that shard obtains it
+ * from its own sampler with the local uniform
+ *   u_local = ceil((y - total of the shards before) 2^64 / T_shard),
+ * for which floor(u_local T_shard / 2^64) is that local threshold exactly.
+ *   shard_totals_device : [n_shards] device array, total mass of every shard in
+ *       order (distrl_sampler_total of each, gathered); n_shards <= 64.
+ *   u_local_out : [k] the local uniform where this shard (my_shard) owns the
+ *       draw, 0 elsewhere;  mine_out : [k] bytes, 1 where it owns the draw;
+ *   owner_out : [k] owning shard of every draw, or NULL.
+ *   status_out_device : device int or NULL; DISTRL_ERR_SIZE if the totals sum
+ *       to 0 or do not fit 64 bits (then nothing is owned).
+ * Every shard then calls distrl_sample with u_local_out as it is and keeps the
+ * positions it owns; un-normalised local weights become global ones by a factor
+ * per shard, ((N / N_shard)(T_shard / T))^-beta.
+ */
+int distrl_route_draws(const uint64_t *u_fix, int64_t k, const uint64_t *shard_totals_device,
+                       int n_shards, int my_shard, uint64_t *u_local_out, uint8_t *mine_out,
+                       int *owner_out, int *status_out_device, void *stream);
+
+/*
+ * What a shard contributes to a batch drawn over several shards, after it has
+ * sampled with distrl_route_draws' uniforms (normalise = 0): for the draws it
+ * owns, the global index index_base + idx_local[j] and the un-normalised global
+ * weight (n_global q / T)^-beta = w_local[j] ((n_global / n_local)(T_shard / T))^-beta;
+ * -1 and 0 for the others, so that an element-wise maximum over the shards (one
+ * all-reduce) assembles the batch.  distrl_normalise_weights then divides the
+ * assembled weights by their maximum, as distrl_sample does for one shard.
+ *   mine, idx_local, w_local : [k] as written by distrl_route_draws / distrl_sample;
+ *   index_base : number of transitions in the shards before this one;
+ *   w_global_out : [k] or NULL (then w_local may be NULL too).
+ */
+int distrl_finish_shard_draws(int64_t k, const uint8_t *mine, const int64_t *idx_local,
+                              const float *w_local, const uint64_t *shard_totals_device,
+                              int n_shards, int my_shard, int64_t n_local, int64_t n_global,
+                              int64_t index_base, float beta, int64_t *idx_global_out,
+                              float *w_global_out, void *stream);
+int distrl_normalise_weights(float *is_weight, int64_t k, void *stream);
+
+/*
  * Priority refresh for sampled indices (Section 5.3: priorities are updated
  * from the latest policy).  For j = 0..k-1 in order:
  *   mass_j = (w_td |new_abs_delta[j]| + w_rho min(rho_i, rho_clip) + w_ent H_i)^alpha,

@@ -114,6 +114,9 @@ def _open(path):
         "distrl_build_sampler": (ci, [vp, i64, vp, sz, vp, ctypes.POINTER(vp)]),
         "distrl_sample": (ci, [vp, vp, i64, f32, ci, vp, vp, vp]),
         "distrl_stratify_uniforms": (ci, [vp, i64, vp, vp]),
+        "distrl_route_draws": (ci, [vp, i64, vp, ci, ci, vp, vp, vp, vp, vp]),
+        "distrl_finish_shard_draws": (ci, [i64, vp, vp, vp, vp, ci, ci, i64, i64, i64, f32, vp, vp, vp]),
+        "distrl_normalise_weights": (ci, [vp, i64, vp]),
         "distrl_update_priorities": (ci, [vp, vp, i64, vp, vp, vp, vp, ctypes.POINTER(distrl_prio_cfg), vp, vp]),
         "distrl_retrace_priorities_build": (ci, [ctypes.POINTER(distrl_batch), f32, f32, vp, vp,
                                                  ctypes.POINTER(distrl_prio_cfg), vp, vp, vp, vp, vp, vp, sz, vp, sz, vp,
@@ -319,6 +322,42 @@ def distrl_stratify_uniforms(u_fix: torch.Tensor, u_out: torch.Tensor, stream=No
         raise ValueError("two arrays of 64-bit fixed-point uniforms of the same length")
     _check(_load().distrl_stratify_uniforms(_ptr(u_fix), u_fix.numel(), _ptr(u_out), _stream(stream)),
            "distrl_stratify_uniforms")
+
+
+def distrl_route_draws(u_fix: torch.Tensor, shard_totals: torch.Tensor, my_shard: int, u_local_out: torch.Tensor,
+                       mine_out: torch.Tensor, owner_out: Optional[torch.Tensor] = None,
+                       status: Optional[torch.Tensor] = None, stream=None):
+    """Global draws over several shards: the local uniform of every draw this shard owns (0 elsewhere) and
+    which draws those are.  shard_totals: device array of the shards' total masses (64-bit), in shard order."""
+    k = u_fix.numel()
+    if u_fix.element_size() != 8 or shard_totals.element_size() != 8 or u_local_out.element_size() != 8:
+        raise ValueError("uniforms and totals are 64-bit integers")
+    if u_local_out.numel() != k or mine_out.numel() != k or mine_out.element_size() != 1:
+        raise ValueError("one local uniform and one byte per draw")
+    if owner_out is not None and (owner_out.numel() != k or owner_out.element_size() != 4):
+        raise ValueError("owner_out holds one 32-bit integer per draw")
+    _check(_load().distrl_route_draws(_ptr(u_fix), k, _ptr(shard_totals), shard_totals.numel(), int(my_shard),
+                                      _ptr(u_local_out), _ptr(mine_out), _ptr(owner_out, torch.int32),
+                                      _ptr(status, torch.int32), _stream(stream)), "distrl_route_draws")
+
+
+def distrl_finish_shard_draws(mine, idx_local, w_local, shard_totals, my_shard: int, n_local: int, n_global: int,
+                              index_base: int, beta: float, idx_global_out, w_global_out=None, stream=None):
+    """Global indices and un-normalised global weights of the draws this shard owns; -1 and 0 elsewhere."""
+    k = idx_local.numel()
+    if mine.numel() != k or idx_global_out.numel() != k or (w_global_out is not None and w_global_out.numel() != k):
+        raise ValueError("one entry per draw")
+    _check(_load().distrl_finish_shard_draws(k, _ptr(mine, torch.uint8), _ptr(idx_local, torch.int64),
+                                             _ptr(w_local, torch.float32), _ptr(shard_totals), shard_totals.numel(),
+                                             int(my_shard), int(n_local), int(n_global), int(index_base), float(beta),
+                                             _ptr(idx_global_out, torch.int64), _ptr(w_global_out, torch.float32),
+                                             _stream(stream)), "distrl_finish_shard_draws")
+
+
+def distrl_normalise_weights(is_weight: torch.Tensor, stream=None):
+    """is_weight /= max(is_weight), in place."""
+    _check(_load().distrl_normalise_weights(_ptr(is_weight, torch.float32), is_weight.numel(), _stream(stream)),
+           "distrl_normalise_weights")
 
 
 def distrl_update_priorities(s: Sampler, idx, new_abs_delta, logp_target, logp_behaviour, entropy,

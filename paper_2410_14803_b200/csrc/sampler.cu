@@ -973,6 +973,152 @@ extern "C" int distrl_stratify_uniforms(const uint64_t *u_fix, int64_t k, uint64
     return DISTRL_OK;
 }
 
+namespace distrl {
+constexpr int kMaxShards = 64;
+// One replay over several shards: draw j has the global threshold y = floor(u[j] T / 2^64), T the total
+// mass of all shards; it belongs to the shard g whose range of cumulative mass holds y, and inside that
+// shard it is the draw with threshold y - (total of the shards before g), which the local uniform
+// ceil((y - before) 2^64 / T_g) reproduces exactly.
+__global__ void route_draws_kernel(const unsigned long long *__restrict__ u, long long k,
+                                   const unsigned long long *__restrict__ totals, int n_shards, int me,
+                                   unsigned long long *__restrict__ u_local, unsigned char *__restrict__ mine,
+                                   int *__restrict__ owner, int *status) {
+    __shared__ unsigned long long s_before[kMaxShards + 1];
+    __shared__ int s_bad;
+    if (threadIdx.x == 0) {
+        unsigned __int128 run = 0;
+        for (int g = 0; g < n_shards; ++g) {
+            s_before[g] = (unsigned long long)run;
+            run += totals[g];
+        }
+        s_before[n_shards] = (unsigned long long)run;
+        s_bad = (run == 0 || (run >> 64) != 0) ? 1 : 0; // nothing to draw from, or a total beyond 64 bits
+    }
+    __syncthreads();
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    if (s_bad) {
+        if (blockIdx.x == 0 && threadIdx.x == 0 && status) set_status(status, DISTRL_ERR_SIZE);
+        for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < k; j += stride) {
+            u_local[j] = 0ull;
+            mine[j] = 0;
+            if (owner) owner[j] = -1;
+        }
+        return;
+    }
+    const unsigned long long grand = s_before[n_shards];
+    for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < k; j += stride) {
+        const unsigned long long y = __umul64hi(u[j], grand); // < grand
+        int g = 0;
+        while (g + 1 < n_shards && s_before[g + 1] <= y) ++g; // few shards: a linear walk (empty shards are passed over)
+        unsigned long long up = 0ull;
+        if (g == me) {
+            const unsigned long long t = s_before[g + 1] - s_before[g], y_local = y - s_before[g]; // y_local < t
+            const unsigned __int128 num = (unsigned __int128)y_local << 64;
+            const unsigned long long quo = (unsigned long long)(num / t);
+            up = quo + ((unsigned __int128)quo * t != num ? 1ull : 0ull); // the ceiling: still below 2^64 since y_local < t
+        }
+        u_local[j] = up;
+        mine[j] = (g == me) ? 1 : 0;
+        if (owner) owner[j] = g;
+    }
+}
+} // namespace distrl
+
+extern "C" int distrl_route_draws(const uint64_t *u_fix, int64_t k, const uint64_t *shard_totals_device, int n_shards,
+                                  int my_shard, uint64_t *u_local_out, uint8_t *mine_out, int *owner_out,
+                                  int *status_out_device, void *stream) {
+    if (k < 0 || k > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
+    if (n_shards < 1 || n_shards > kMaxShards || my_shard < 0 || my_shard >= n_shards) return DISTRL_ERR_PARAM;
+    if (k == 0) return DISTRL_OK;
+    if (!u_fix || !shard_totals_device || !u_local_out || !mine_out) return DISTRL_ERR_NULL;
+    if (!aligned_to(u_fix, 8) || !aligned_to(shard_totals_device, 8) || !aligned_to(u_local_out, 8) ||
+        !aligned_to(owner_out, 4) || !aligned_to(status_out_device, 4))
+        return DISTRL_ERR_ALIGN;
+    int64_t grid = ceil_div(k, 256);
+    if (grid > 1184) grid = 1184;
+    route_draws_kernel<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<const unsigned long long *>(u_fix), (long long)k,
+        reinterpret_cast<const unsigned long long *>(shard_totals_device), n_shards, my_shard,
+        reinterpret_cast<unsigned long long *>(u_local_out), mine_out, owner_out, status_out_device);
+    DISTRL_CUDA_TRY(cudaGetLastError());
+    return DISTRL_OK;
+}
+
+namespace distrl {
+// What a shard contributes to a batch drawn over several shards: for the draws it owns, the global index
+// and the un-normalised global weight (N q / T)^-beta = (N_shard q / T_shard)^-beta x ((N / N_shard)(T_shard / T))^-beta;
+// -1 and 0 elsewhere, so that an element-wise maximum over the shards assembles the batch.
+__global__ void finish_shard_draws_kernel(long long k, const unsigned char *__restrict__ mine,
+                                          const long long *__restrict__ idx_local, const float *__restrict__ w_local,
+                                          const unsigned long long *__restrict__ totals, int n_shards, int me,
+                                          long long n_local, long long n_global, long long index_base, float beta,
+                                          long long *__restrict__ idx_out, float *__restrict__ w_out) {
+    double grand = 0.0;
+    for (int g = 0; g < n_shards; ++g) grand += (double)totals[g];
+    const double ratio = ((double)n_global / (double)n_local) * ((double)totals[me] / grand);
+    const float factor = (float)pow(ratio, -(double)beta);
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < k; j += stride) {
+        const bool own = mine[j] != 0 && idx_local[j] >= 0;
+        idx_out[j] = own ? index_base + idx_local[j] : -1;
+        if (w_out) w_out[j] = own ? w_local[j] * factor : 0.f;
+    }
+}
+
+// w[j] /= max_j w[j] (one block; the batch maximum of Section 5.3's importance weights)
+__global__ void __launch_bounds__(1024) normalise_weights_kernel(float *__restrict__ w, long long k) {
+    __shared__ float s_max[32];
+    float m = 0.f;
+    for (long long j = threadIdx.x; j < k; j += blockDim.x) m = fmaxf(m, w[j]);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+    if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    m = (threadIdx.x < 32) ? s_max[threadIdx.x] : 0.f;
+    if (threadIdx.x < 32) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+        if (threadIdx.x == 0) s_max[0] = m;
+    }
+    __syncthreads();
+    m = s_max[0];
+    if (!(m > 0.f)) return; // no weight at all: leave the zeros
+    for (long long j = threadIdx.x; j < k; j += blockDim.x) w[j] = w[j] / m;
+}
+} // namespace distrl
+
+extern "C" int distrl_finish_shard_draws(int64_t k, const uint8_t *mine, const int64_t *idx_local, const float *w_local,
+                                         const uint64_t *shard_totals_device, int n_shards, int my_shard,
+                                         int64_t n_local, int64_t n_global, int64_t index_base, float beta,
+                                         int64_t *idx_global_out, float *w_global_out, void *stream) {
+    if (k < 0 || k > DISTRL_MAX_N || n_local <= 0 || n_global < n_local || index_base < 0) return DISTRL_ERR_SIZE;
+    if (n_shards < 1 || n_shards > kMaxShards || my_shard < 0 || my_shard >= n_shards || !(beta == beta))
+        return DISTRL_ERR_PARAM;
+    if (k == 0) return DISTRL_OK;
+    if (!mine || !idx_local || !shard_totals_device || !idx_global_out || (w_global_out && !w_local)) return DISTRL_ERR_NULL;
+    if (!aligned_to(idx_local, 8) || !aligned_to(idx_global_out, 8) || !aligned_to(shard_totals_device, 8) ||
+        !aligned_to(w_local, 4) || !aligned_to(w_global_out, 4))
+        return DISTRL_ERR_ALIGN;
+    int64_t grid = ceil_div(k, 256);
+    if (grid > 1184) grid = 1184;
+    finish_shard_draws_kernel<<<(unsigned)grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        (long long)k, mine, reinterpret_cast<const long long *>(idx_local), w_local,
+        reinterpret_cast<const unsigned long long *>(shard_totals_device), n_shards, my_shard, (long long)n_local,
+        (long long)n_global, (long long)index_base, beta, reinterpret_cast<long long *>(idx_global_out), w_global_out);
+    DISTRL_CUDA_TRY(cudaGetLastError());
+    return DISTRL_OK;
+}
+
+extern "C" int distrl_normalise_weights(float *is_weight, int64_t k, void *stream) {
+    if (k < 0 || k > DISTRL_MAX_N) return DISTRL_ERR_SIZE;
+    if (k == 0) return DISTRL_OK;
+    if (!is_weight) return DISTRL_ERR_NULL;
+    if (!aligned_to(is_weight, 4)) return DISTRL_ERR_ALIGN;
+    normalise_weights_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(is_weight, (long long)k);
+    DISTRL_CUDA_TRY(cudaGetLastError());
+    return DISTRL_OK;
+}
+
 extern "C" int distrl_sampler_total(distrl_sampler *s, uint64_t *total_out_device, void *stream) {
     if (!s || !total_out_device) return DISTRL_ERR_NULL;
     if (!aligned_to(total_out_device, 8)) return DISTRL_ERR_ALIGN;

@@ -545,6 +545,93 @@ def test_draws_over_two_shards_through_the_ordinary_entry_point():
     sb.close()
 
 
+def test_draws_routed_on_the_device_over_three_shards():
+    # the same routing done by distrl_route_draws from a device array of the shards' totals: every shard samples
+    # all k positions with what the call gives it and keeps the ones it owns; together they are one linear scan
+    # over the concatenated masses.  The local uniforms equal the host routine's, the owners the plain definition.
+    from paper_2410_14803_b200 import shard, binding
+    qs = [_masses(200_001, 41), np.array([7], dtype=np.uint32), _masses(123_457, 42, heavy=False)]
+    built = [_build(q) for q in qs]
+    totals = [int(q.sum(dtype=np.uint64)) for q in qs]
+    d_tot = torch.zeros(3, dtype=torch.int64, device="cuda")
+    for g, (s, _, _) in enumerate(built):
+        distrl.distrl_sampler_total(s, d_tot[g:g + 1])
+    torch.cuda.synchronize()
+    assert [int(x) for x in d_tot.cpu().numpy().view(np.uint64)] == totals
+    k = 5000
+    u = np.random.default_rng(43).integers(0, 2 ** 64, size=k, dtype=np.uint64)
+    u[:4] = [0, 2 ** 64 - 1, 1, 2 ** 63]
+    grand = sum(totals)
+    ys = [(int(x) * grand) >> 64 for x in u]
+    u[4] = -((-(totals[0] << 64)) // grand)                    # the first threshold of the one-mass shard ...
+    u[5] = -((-((totals[0] + 6) << 64)) // grand)              # ... and its last
+    u[6] = -((-((totals[0] + 7) << 64)) // grand)              # the first of the third shard
+    ys = [(int(x) * grand) >> 64 for x in u]
+    assert ys[4] == totals[0] and ys[5] == totals[0] + 6 and ys[6] == totals[0] + 7
+    d_u = dev(u.view(np.int64))
+    owner_host, ul_host = shard.route_draws(u.tolist(), totals)
+    before = np.concatenate([[0], np.cumsum(np.array(totals, dtype=object))])
+    got = np.full(k, -1, dtype=np.int64)
+    base, n_all, parts_i, parts_w = 0, sum(q.shape[0] for q in qs), [], []
+    for g, (s, _, ws) in enumerate(built):
+        ul = torch.empty(k, dtype=torch.int64, device="cuda")
+        mine = torch.empty(k, dtype=torch.uint8, device="cuda")
+        owner = torch.empty(k, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        distrl.distrl_route_draws(d_u, d_tot, g, ul, mine, owner, status)
+        idx = torch.empty(k, dtype=torch.int64, device="cuda")
+        wts = torch.empty(k, dtype=torch.float32, device="cuda")
+        distrl.distrl_sample(s, ul, 0.4, False, idx, wts)
+        torch.cuda.synchronize()
+        assert status.item() == 0 and distrl.distrl_get_status(ws) == 0
+        m = mine.cpu().numpy().astype(bool)
+        ow = owner.cpu().numpy()
+        assert ow.tolist() == owner_host
+        assert [bool(x) for x in m] == [o == g for o in owner_host]
+        assert all(before[o] <= y < before[o + 1] for o, y in zip(ow, ys))
+        ulh = ul.cpu().numpy().view(np.uint64)
+        assert [int(x) for x in ulh[m]] == [ul_host[j] for j in np.nonzero(m)[0]]
+        assert np.all(ulh[~m] == 0)
+        got[m] = base + idx.cpu().numpy()[m]
+        # the shard's contribution to the batch: global indices and un-normalised global weights, -1 / 0 elsewhere
+        gi = torch.empty(k, dtype=torch.int64, device="cuda")
+        gw = torch.empty(k, dtype=torch.float32, device="cuda")
+        distrl.distrl_finish_shard_draws(mine, idx, wts, d_tot, g, qs[g].shape[0], n_all, base, 0.4, gi, gw)
+        torch.cuda.synchronize()
+        parts_i.append(gi.cpu().numpy())
+        parts_w.append(gw.cpu().numpy())
+        assert np.all(parts_i[-1][~m] == -1) and np.all(parts_w[-1][~m] == 0)
+        base += qs[g].shape[0]
+    q_all = np.concatenate(qs)
+    np.testing.assert_array_equal(got, sample_by_prefix(q_all, u))
+    # an element-wise maximum over the shards (what one all-reduce does) assembles the batch
+    all_i, all_w = np.maximum.reduce(parts_i), np.maximum.reduce(parts_w)
+    np.testing.assert_array_equal(all_i, got)
+    assert_close(all_w, oracle.is_weights(q_all, got, 0.4, False), "global un-normalised weights")
+    d_w = dev(all_w)
+    distrl.distrl_normalise_weights(d_w)
+    torch.cuda.synchronize()
+    assert_close(d_w.cpu().numpy(), oracle.is_weights(q_all, got, 0.4, True), "global weights / batch maximum")
+    assert d_w.max().item() == 1.0
+    # totals that do not fit 64 bits, or no mass at all: reported, nothing owned
+    for bad in ([2 ** 63, 2 ** 63, 5], [0, 0, 0]):
+        d_bad = dev(np.array(bad, dtype=np.uint64).view(np.int64))
+        ul = torch.full((k,), 9, dtype=torch.int64, device="cuda")
+        mine = torch.full((k,), 9, dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        distrl.distrl_route_draws(d_u, d_bad, 1, ul, mine, None, status)
+        torch.cuda.synchronize()
+        assert status.item() == binding.ERR_SIZE
+        assert int(ul.abs().sum().item()) == 0 and int(mine.sum().item()) == 0
+    lib = binding._load()
+    assert lib.distrl_route_draws(d_u.data_ptr(), k, d_tot.data_ptr(), 0, 0, ul.data_ptr(), mine.data_ptr(), None, None, None) == binding.ERR_PARAM
+    assert lib.distrl_route_draws(d_u.data_ptr(), k, d_tot.data_ptr(), 3, 3, ul.data_ptr(), mine.data_ptr(), None, None, None) == binding.ERR_PARAM
+    assert lib.distrl_route_draws(d_u.data_ptr(), k, None, 3, 0, ul.data_ptr(), mine.data_ptr(), None, None, None) == binding.ERR_NULL
+    assert lib.distrl_route_draws(None, 0, None, 3, 0, None, None, None, None, None) == binding.OK
+    for s, _, _ in built:
+        s.close()
+
+
 @pytest.mark.parametrize("k", [1, 2, 3, 255, 4096, 100_003])
 def test_stratified_uniforms_and_a_stratified_batch(k):
     rng = np.random.default_rng(k)
