@@ -74,3 +74,41 @@ def global_weight_factor(n_local: int, total_local: int, n_global: int, total_gl
     """What a shard multiplies its un-normalised local importance weights (n_local q / T_local)^-beta by to get
     the global ones (n_global q / T_global)^-beta; the batch maximum is then one all-reduce (max_over_ranks)."""
     return ((n_global / n_local) * (total_local / total_global)) ** (-beta)
+
+
+def sample_over_shards(sampler, n_local: int, u_fix, beta: float, idx_out, w_out, normalise: bool = True):
+    """One batch drawn over all ranks' shards, every step on the device (device tensors in and out).
+
+    All-gathers the shards' totals and sizes, routes the draws (distrl_route_draws), samples locally with
+    the routed uniforms, turns the owned draws into global indices and weights (distrl_finish_shard_draws),
+    assembles the batch with one element-wise maximum over the ranks and divides by the batch maximum.
+    With one rank it is distrl_sample with a detour."""
+    from . import binding as b
+    k = u_fix.numel()
+    dev = u_fix.device
+    world = dist.get_world_size() if (dist.is_available() and dist.is_initialized()) else 1
+    rank = dist.get_rank() if world > 1 else 0
+    mine_total = torch.zeros(1, dtype=torch.int64, device=dev)
+    b.distrl_sampler_total(sampler, mine_total)
+    sizes = torch.tensor([int(n_local)], dtype=torch.int64, device=dev)
+    if world > 1:
+        totals = torch.zeros(world, dtype=torch.int64, device=dev)
+        all_n = torch.zeros(world, dtype=torch.int64, device=dev)
+        dist.all_gather_into_tensor(totals, mine_total)
+        dist.all_gather_into_tensor(all_n, sizes)
+        ns = [int(x) for x in all_n.cpu()]
+    else:
+        totals, ns = mine_total, [int(n_local)]
+    u_local = torch.empty(k, dtype=torch.int64, device=dev)
+    mine = torch.empty(k, dtype=torch.uint8, device=dev)
+    b.distrl_route_draws(u_fix, totals, rank, u_local, mine)
+    idx_local = torch.empty(k, dtype=torch.int64, device=dev)
+    w_local = torch.empty(k, dtype=torch.float32, device=dev)
+    b.distrl_sample(sampler, u_local, beta, False, idx_local, w_local)
+    b.distrl_finish_shard_draws(mine, idx_local, w_local, totals, rank, ns[rank], sum(ns), sum(ns[:rank]), beta,
+                                idx_out, w_out)
+    if world > 1:
+        dist.all_reduce(idx_out, op=dist.ReduceOp.MAX)
+        dist.all_reduce(w_out, op=dist.ReduceOp.MAX)
+    if normalise:
+        b.distrl_normalise_weights(w_out)

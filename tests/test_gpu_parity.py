@@ -632,6 +632,21 @@ def test_draws_routed_on_the_device_over_three_shards():
         s.close()
 
 
+def test_sample_over_shards_with_one_rank_is_the_ordinary_draw():
+    from paper_2410_14803_b200 import shard
+    q = _masses(77_777, 51)
+    s, tq, ws = _build(q)
+    u = np.random.default_rng(52).integers(0, 2 ** 64, size=2000, dtype=np.uint64)
+    idx = torch.empty(2000, dtype=torch.int64, device="cuda")
+    wts = torch.empty(2000, dtype=torch.float32, device="cuda")
+    shard.sample_over_shards(s, q.shape[0], dev(u.view(np.int64)), 0.4, idx, wts)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(idx.cpu().numpy(), sample_by_prefix(q, u))
+    assert_close(wts.cpu().numpy(), oracle.is_weights(q, idx.cpu().numpy(), 0.4, True), "weights")
+    assert distrl.distrl_get_status(ws) == 0
+    s.close()
+
+
 @pytest.mark.parametrize("k", [1, 2, 3, 255, 4096, 100_003])
 def test_stratified_uniforms_and_a_stratified_batch(k):
     rng = np.random.default_rng(k)
