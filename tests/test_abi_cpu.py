@@ -99,6 +99,18 @@ def test_argument_validation_happens_before_any_device_work():
     assert lib.distrl_replay_head(None) == -1 and lib.distrl_replay_destroy(None) == 0
     assert distrl.distrl_replay_workspace_bytes(1 << 24) == 256 + 2 * (1 << 21) + 256 * ((513 * 8 + 255) // 256)
     assert lib.distrl_set_cooperative_launch(1) == 1
+    # draws over several shards
+    assert lib.distrl_route_draws(None, 1, None, 0, 0, None, None, None, None, None) == binding.ERR_PARAM
+    assert lib.distrl_route_draws(None, 1, None, 65, 0, None, None, None, None, None) == binding.ERR_PARAM
+    assert lib.distrl_route_draws(None, 1, None, 2, 2, None, None, None, None, None) == binding.ERR_PARAM
+    assert lib.distrl_route_draws(None, 1, None, 2, 1, None, None, None, None, None) == binding.ERR_NULL
+    assert lib.distrl_route_draws(None, 0, None, 2, 1, None, None, None, None, None) == binding.OK
+    assert lib.distrl_finish_shard_draws(1, None, None, None, None, 2, 0, 0, 10, 0, 0.4, None, None, None) == binding.ERR_SIZE
+    assert lib.distrl_finish_shard_draws(1, None, None, None, None, 2, 0, 20, 10, 0, 0.4, None, None, None) == binding.ERR_SIZE
+    assert lib.distrl_finish_shard_draws(1, None, None, None, None, 2, 2, 5, 10, 0, 0.4, None, None, None) == binding.ERR_PARAM
+    assert lib.distrl_finish_shard_draws(1, None, None, None, None, 2, 0, 5, 10, 0, 0.4, None, None, None) == binding.ERR_NULL
+    assert lib.distrl_normalise_weights(None, 0, None) == binding.OK
+    assert lib.distrl_normalise_weights(None, 3, None) == binding.ERR_NULL
 
 
 def test_binding_refuses_host_tensors():
